@@ -1,0 +1,252 @@
+/*
+ * avmp.h -- C ABI of the B200-native AVMP hot path.
+ *
+ * AVMP (Asymmetric Virtual Memory Paging) keeps two physically different cache
+ * stores for hybrid Mamba-Transformer inference -- fine-grained KV pages and
+ * per-layer SSM state blocks -- behind one space of 32-bit virtual handles, and
+ * moves capacity between them when an allocation would otherwise fail (paper
+ * Sections 3.1 and 3.2).  This library holds all allocator state in device
+ * memory and runs every step of the path as CUDA kernels on sm_100a:
+ *
+ *   avmp_step        batched admit / extend / finish in array order, including the
+ *                    CapacityError handler, the migration (shrink donor, relocate
+ *                    live units, remap handles, grow recipient) and the retry;
+ *   avmp_translate   handle -> (pool, physical offset);
+ *   avmp_gather_kv   paged gather of one attention layer into ragged batch buffers;
+ *   avmp_gather_ssm  gather of one SSM layer's state blocks into batch buffers;
+ *   avmp_scatter_*   the matching write side.
+ *
+ * Conventions
+ *   - "d_" arguments are DEVICE pointers, "h_" arguments are HOST pointers.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Every call is ordered on that stream.  Calls with only device arguments never
+ *     synchronise with the host; calls that take or fill host memory do, and say so.
+ *   - The library never allocates device memory: the caller owns the arena and the
+ *     workspace (e.g. two torch tensors) and must keep them alive until avmp_destroy.
+ *   - Return value: AVMP_OK or a negative AVMP_E* code for misuse the host can see.
+ *     What only the device can see (an invalid handle, a dead request in a gather
+ *     list, an output buffer too small) never traps: the item is skipped, a sticky
+ *     error code and an error count are recorded in the statistics block.
+ *   - One context must not be used from two streams at once.
+ */
+#ifndef AVMP_H
+#define AVMP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define AVMP_API __attribute__((visibility("default")))
+#else
+#define AVMP_API
+#endif
+
+#define AVMP_INVALID 0xFFFFFFFFu              /* no handle / no slot */
+#define AVMP_NONE64 0xFFFFFFFFFFFFFFFFull     /* no offset / "never" */
+
+enum { AVMP_OK = 0, AVMP_EINVAL = -1, AVMP_ENOSPC = -2, AVMP_ECUDA = -3 };
+enum { AVMP_POOL_KV = 0, AVMP_POOL_SSM = 1 };
+
+/* Operation kinds and flags (avmp_op). */
+enum { AVMP_OP_ADMIT = 1, AVMP_OP_EXTEND = 2, AVMP_OP_FINISH = 3 };
+enum {
+    AVMP_FLAG_KEEP_KV = 1, /* FINISH: free only the SSM blocks, keep the KV chain (slot becomes KV_ONLY) */
+    AVMP_FLAG_RESUME = 2   /* ADMIT: the slot is KV_ONLY; allocate SSM blocks and extend the kept chain */
+};
+/* Per-operation result written by avmp_step. */
+enum {
+    AVMP_ST_OK = 0,
+    AVMP_ST_OOM = 1,      /* did not fit, even after the migration attempt; nothing was taken */
+    AVMP_ST_BAD_REQ = 2,  /* slot out of range or in the wrong state for this kind */
+    AVMP_ST_TOO_LONG = 3, /* chain would pass max_pages_per_request */
+    AVMP_ST_BAD_ARG = 4   /* unknown kind, or zero tokens on ADMIT / EXTEND */
+};
+enum { AVMP_REQ_EMPTY = 0, AVMP_REQ_LIVE = 1, AVMP_REQ_KV_ONLY = 2 };
+/* Rebalancer state label (paper Figure 2). */
+enum { AVMP_FSM_BALANCED = 0, AVMP_FSM_KV_PRESSURED = 1, AVMP_FSM_SSM_PRESSURED = 2, AVMP_FSM_REBALANCING = 3 };
+/* Sticky device-side error codes (avmp_stats.error_code keeps the first one). */
+enum {
+    AVMP_DEV_OK = 0,
+    AVMP_DEV_BAD_HANDLE = 1,     /* translate: handle does not resolve */
+    AVMP_DEV_BAD_REQUEST = 2,    /* gather / scatter: request slot out of range or holds nothing */
+    AVMP_DEV_OUT_OVERFLOW = 3    /* gather_kv: rows would pass out_capacity_tokens */
+};
+
+/* Model shape: what one KV page and one SSM block hold (paper Section 3.1).
+ * KV page  = page_tokens tokens of {K, V} x kv_heads x head_dim x kv_elem_bytes for EVERY
+ *            attention layer, laid out [layer][K|V][token][head][dim];
+ * SSM block = one layer's ssm_state_elems then ssm_conv_elems elements of ssm_elem_bytes. */
+typedef struct {
+    uint32_t n_attn_layers, n_ssm_layers, page_tokens, kv_heads, head_dim, kv_elem_bytes;
+    uint32_t ssm_state_elems, ssm_conv_elems, ssm_elem_bytes;
+} avmp_model_spec;
+
+/* Rebalancer and table-size options (paper Section 3.2; defaults from avmp_default_options). */
+typedef struct {
+    uint32_t threshold_low_ppm;           /* 50000: labels the PRESSURED states only */
+    uint32_t threshold_high_ppm;          /* 300000: donor free fraction must exceed this */
+    uint64_t min_rebalance_interval_ops;  /* 1000 logical operations between migrations; >= 1 */
+    uint32_t migration_enabled;           /* 0 = static partition with AVMP handles */
+    uint32_t max_requests;                /* request slots: op.req is in [0, max_requests) */
+    uint32_t max_pages_per_request;       /* longest KV chain, in pages */
+} avmp_options;
+
+/* One allocator operation, 12 bytes. */
+typedef struct {
+    uint8_t kind, flags;
+    uint16_t rsvd;
+    uint32_t req;     /* caller-chosen dense slot id */
+    uint32_t tokens;  /* ADMIT / EXTEND: tokens appended */
+} avmp_op;
+
+/* Sizes derived from the model and the pool (host-side arithmetic, no device access). */
+typedef struct {
+    uint64_t pool_bytes_aligned;  /* pool_bytes rounded down to 128 (slab alignment) */
+    uint64_t unit_bytes[2];       /* KV page, SSM block; each rounded up to 16 */
+    uint64_t vid_space[2];        /* virtual ids per pool = pool_bytes_aligned / unit */
+    uint64_t cap0[2];             /* initial capacities in units */
+    uint64_t gap0;                /* initial bytes in neither store */
+    uint64_t kv_layer_bytes;      /* one attention layer inside a page (K then V) */
+    uint64_t kv_row_bytes;        /* one token's K (or V) of one layer */
+    uint64_t ssm_state_bytes, ssm_conv_bytes;
+} avmp_layout;
+
+/* All counters of a context (same order as uint64_t[AVMP_N_STATS]). */
+typedef struct {
+    uint64_t op_counter;          /* logical operations processed (Section 3.2) */
+    uint64_t last_rebalance_op;   /* AVMP_NONE64 before the first migration */
+    uint64_t n_oom;               /* operations that ended AVMP_ST_OOM (the paper's N_OOM) */
+    uint64_t n_capacity_error;    /* CapacityError handler runs */
+    uint64_t n_rebalance;         /* completed migrations */
+    uint64_t migrated_bytes;      /* donor bytes ceded */
+    uint64_t wasted_bytes;        /* sum of ceded bytes modulo the recipient unit */
+    uint64_t relocated_blocks;    /* live units copied out of ceded regions */
+    uint64_t relocated_bytes;
+    uint64_t gap_bytes;
+    uint64_t cap[2];
+    uint64_t free_units[2];
+    uint64_t fsm_state;
+    uint64_t n_invalid;           /* operations rejected with BAD_REQ / TOO_LONG / BAD_ARG */
+    uint64_t unit_bytes[2];
+    uint64_t vid_space[2];
+    uint64_t pool_bytes_aligned;
+    uint64_t error_code;          /* first AVMP_DEV_* error seen, sticky */
+    uint64_t error_count;         /* items skipped because of device-side errors */
+} avmp_stats;
+#define AVMP_N_STATS (sizeof(avmp_stats) / sizeof(uint64_t))
+
+/* Host copies of every table, for parity checks and snapshot / restore.  The caller
+ * provides the arrays (sizes from avmp_layout and avmp_options); counts are filled by
+ * export and read by import. */
+typedef struct {
+    uint32_t *slot_stack[2];  /* [vid_space[p]]  free physical slots, bottom first */
+    uint32_t *vid_stack[2];   /* [vid_space[p]]  free virtual ids, bottom first */
+    uint32_t *vt[2];          /* [vid_space[p]]  page table: vid -> slot or AVMP_INVALID */
+    uint32_t *ow[2];          /* [vid_space[p]]  owner: slot -> vid or AVMP_INVALID */
+    uint32_t *req_state;      /* [max_requests] */
+    uint32_t *req_len;        /* [max_requests] tokens held */
+    uint32_t *req_npages;     /* [max_requests] */
+    uint32_t *req_chain;      /* [max_requests * max_pages_per_request] KV handles */
+    uint32_t *req_ssm;        /* [max_requests * n_ssm_layers] SSM handles */
+    uint32_t n_slot_stack[2], n_vid_stack[2];
+    avmp_stats stats;
+} avmp_tables;
+
+typedef struct avmp_ctx avmp_ctx;
+
+/* Fill *opt with the paper's defaults (thresholds 0.05 / 0.30, interval 1000, migration
+ * on) and max_requests = 1024, max_pages_per_request = 4096. */
+AVMP_API void avmp_default_options(avmp_options *opt);
+
+/* Section 3.1 arithmetic.  initial_split is the fraction of the pool given to the SSM store
+ * at start (the static systems' "mamba ratio").  Returns AVMP_EINVAL on zero units, a split
+ * outside [0, 1], a pool too small for one unit, or an id space beyond 31 bits. */
+AVMP_API int avmp_derive_layout(const avmp_model_spec *spec, uint64_t pool_bytes, double initial_split,
+                       avmp_layout *out);
+
+/* Bytes of workspace avmp_create needs (0 on invalid arguments). */
+AVMP_API size_t avmp_workspace_bytes(const avmp_model_spec *spec, uint64_t pool_bytes, const avmp_options *opt);
+
+/* Create a context over a caller-owned arena and workspace and initialise the tables on
+ * `stream` (fresh pools hand out slot 0, 1, 2, ... and id 0, 1, 2, ...).
+ *   d_arena      >= pool_bytes, 256-byte aligned.  KV slot i lives at byte i * U_kv; SSM slot j
+ *                at pool_bytes_aligned - (j + 1) * U_ssm, so each store's high end faces the gap
+ *                in the middle and ceded bytes are what the other store grows into.  The arena
+ *                is never cleared.
+ *   d_workspace  >= avmp_workspace_bytes(...), 256-byte aligned.
+ *   migration_batch_size  B: upper bound, in donor units, on one migration (Section 3.1).
+ *   opt          NULL = defaults.  threshold_low >= threshold_high is rejected (Section 4.6).
+ * Returns AVMP_EINVAL / AVMP_ENOSPC (workspace too small) / AVMP_ECUDA. */
+AVMP_API int avmp_create(avmp_ctx **out, const avmp_model_spec *spec, void *d_arena, uint64_t pool_bytes,
+                double initial_split, uint32_t migration_batch_size, const avmp_options *opt,
+                void *d_workspace, size_t workspace_bytes, void *stream);
+AVMP_API int avmp_destroy(avmp_ctx *ctx);
+
+/* One engine step (Sections 3.1-3.2): process d_ops[0..n_ops) exactly as if they were applied
+ * one at a time in array order -- each op advances the logical counter, allocations pop the
+ * LIFO free lists, a shortage runs the CapacityError handler (SSM first, then KV), which may
+ * migrate min(B, donor free) donor units when the donor's free fraction exceeds
+ * threshold_high and the throttle allows, relocating live units out of the ceded range and
+ * remapping their handles; the op is then retried once.  d_status[i] receives AVMP_ST_*.
+ * Stream-ordered, no host synchronisation.  n_ops == 0 is a no-op. */
+AVMP_API int avmp_step(avmp_ctx *ctx, const avmp_op *d_ops, uint32_t n_ops, uint32_t *d_status, void *stream);
+
+/* Same step with HOST arrays: copies the ops in, runs the step, copies the statuses out
+ * and waits for them.  n_ops is limited to 65536 per call. */
+AVMP_API int avmp_step_host(avmp_ctx *ctx, const avmp_op *h_ops, uint32_t n_ops, uint32_t *h_status, void *stream);
+
+/* Section 3.1 / Figure 1: resolve handles.  d_pool[i] = pool tag, d_offset[i] = slot * unit
+ * bytes (offset inside that store), d_arena_offset[i] (may be NULL) = byte offset of the unit
+ * from d_arena.  A handle that does not resolve gives AVMP_INVALID / AVMP_NONE64 and a sticky
+ * AVMP_DEV_BAD_HANDLE. */
+AVMP_API int avmp_translate(avmp_ctx *ctx, const uint32_t *d_handles, uint32_t n, uint32_t *d_pool,
+                   uint64_t *d_offset, uint64_t *d_arena_offset, void *stream);
+
+/* Paged KV gather (Section 2.2 "paged scatter-gather memory lookups") of attention layer
+ * `attn_layer` for the request slots d_reqs[0..n_reqs), n_reqs <= max_requests.  Rows are one
+ * token's kv_heads x head_dim elements; request k's rows start at d_cu_seqlens[k] (prefix sums
+ * of the held lengths, n_reqs + 1 entries, always written).  Only valid tokens are copied
+ * (the last page may be partial).  A slot that holds no chain contributes length 0 and a
+ * sticky AVMP_DEV_BAD_REQUEST; a request whose rows would pass out_capacity_tokens copies
+ * nothing (AVMP_DEV_OUT_OVERFLOW).  Output pointers must be 16-byte aligned. */
+AVMP_API int avmp_gather_kv(avmp_ctx *ctx, uint32_t attn_layer, const uint32_t *d_reqs, uint32_t n_reqs,
+                   void *d_out_k, void *d_out_v, uint64_t out_capacity_tokens,
+                   uint32_t *d_cu_seqlens, void *stream);
+
+/* SSM gather (Section 2.2 "contiguous read and write access") of SSM layer `ssm_layer`:
+ * d_out_state[k] gets the state elements, d_out_conv[k] the convolution window of request
+ * d_reqs[k].  Requests must be LIVE; others are skipped with AVMP_DEV_BAD_REQUEST. */
+AVMP_API int avmp_gather_ssm(avmp_ctx *ctx, uint32_t ssm_layer, const uint32_t *d_reqs, uint32_t n_reqs,
+                    void *d_out_state, void *d_out_conv, void *stream);
+
+/* Write side of the two gathers (what the model's kernels do after a step).  Tokens
+ * [d_tok_start[k], len_k) of request k are read from rows cu[k].. of d_in_k / d_in_v, cu being
+ * the prefix sum of (len_k - d_tok_start[k]); d_tok_start == NULL means 0. */
+AVMP_API int avmp_scatter_kv(avmp_ctx *ctx, uint32_t attn_layer, const uint32_t *d_reqs,
+                    const uint32_t *d_tok_start, uint32_t n_reqs, const void *d_in_k,
+                    const void *d_in_v, void *stream);
+AVMP_API int avmp_scatter_ssm(avmp_ctx *ctx, uint32_t ssm_layer, const uint32_t *d_reqs, uint32_t n_reqs,
+                     const void *d_in_state, const void *d_in_conv, void *stream);
+
+/* Counters -> host.  Synchronises the stream. */
+AVMP_API int avmp_get_stats(avmp_ctx *ctx, avmp_stats *h_out, void *stream);
+/* Clear the sticky device error code and count.  Stream-ordered. */
+AVMP_API int avmp_clear_error(avmp_ctx *ctx, void *stream);
+
+/* Tables <-> host (parity checks, snapshot / restore).  Both synchronise the stream. */
+AVMP_API int avmp_export_tables(avmp_ctx *ctx, avmp_tables *h_out, void *stream);
+AVMP_API int avmp_import_tables(avmp_ctx *ctx, const avmp_tables *h_in, void *stream);
+
+/* How many kernels this context has launched so far (host counter). */
+AVMP_API uint64_t avmp_launch_count(const avmp_ctx *ctx);
+
+AVMP_API const char *avmp_error_string(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

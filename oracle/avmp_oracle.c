@@ -339,7 +339,7 @@ uint32_t orc_gather_kv(const orc_ctx *c, uint32_t layer, const uint32_t *reqs, u
         uint32_t r = reqs[k];
         uint32_t len = holds_kv(c, r) ? c->r_len[r] : 0;
         if (!holds_kv(c, r)) ++bad;
-        else if (cu + len > capacity_tokens) ++bad;
+        else if (len > 0 && cu + len > capacity_tokens) ++bad;   /* no rows, nothing to overflow */
         else
             for (uint32_t t = 0; t < len; ++t) {
                 memcpy((uint8_t *)out_k + (cu + t) * row, kv_row(c, r, layer, 0, t), row);

@@ -1,0 +1,388 @@
+// Host side of the C ABI: argument checks, the Section 3.1 layout arithmetic, workspace
+// carving, launch sequencing.  No device memory is allocated here; the context is a small
+// host struct over the caller's arena and workspace.
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "avmp_dev.cuh"
+
+using namespace avmp;
+
+struct avmp_ctx {
+    Geom g;
+    avmp_model_spec spec;
+    avmp_options opt;
+    avmp_layout lay;
+    uint32_t B;
+    int n_sms;
+    uint64_t launches;
+    // staging for avmp_step_host, inside the workspace
+    avmp_op *d_stage_ops;
+    uint32_t *d_stage_status;
+    size_t workspace_bytes;
+    void *d_workspace;
+};
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct Carve {
+    size_t off = 0;
+    size_t take(size_t bytes) { size_t o = off; off += up(bytes ? bytes : 1); return o; }
+};
+
+// Offsets of every table inside the workspace, in one place so that size and carving agree.
+struct WsLayout {
+    size_t state, S[2], W[2], VT[2], OW[2], r_state, r_len, r_npages, r_chain, r_ssm, mark;
+    size_t reloc_src, reloc_dst, g_cu_items, g_cu_rows, stage_ops, stage_status, total;
+};
+
+WsLayout ws_layout(const avmp_layout &lay, const avmp_model_spec &spec, const avmp_options &opt)
+{
+    WsLayout w;
+    Carve c;
+    w.state = c.take(sizeof(DevState));
+    for (int p = 0; p < 2; ++p) {
+        const size_t v = (size_t)lay.vid_space[p] * 4;
+        w.S[p] = c.take(v); w.W[p] = c.take(v); w.VT[p] = c.take(v); w.OW[p] = c.take(v);
+    }
+    const size_t R = opt.max_requests;
+    w.r_state = c.take(R * 4); w.r_len = c.take(R * 4); w.r_npages = c.take(R * 4);
+    w.r_chain = c.take(R * (size_t)opt.max_pages_per_request * 4);
+    w.r_ssm = c.take(R * (size_t)spec.n_ssm_layers * 4);
+    w.mark = c.take(R * 4);
+    const size_t maxv = (size_t)(lay.vid_space[0] > lay.vid_space[1] ? lay.vid_space[0] : lay.vid_space[1]);
+    w.reloc_src = c.take(maxv * 4); w.reloc_dst = c.take(maxv * 4);
+    w.g_cu_items = c.take((R + 1) * 4); w.g_cu_rows = c.take((R + 1) * 4);
+    w.stage_ops = c.take((size_t)kHostStepMaxOps * sizeof(avmp_op));
+    w.stage_status = c.take((size_t)kHostStepMaxOps * 4);
+    w.total = c.off;
+    return w;
+}
+
+bool options_ok(const avmp_options &o)
+{
+    return o.threshold_low_ppm < o.threshold_high_ppm && o.threshold_high_ppm <= 1000000u &&
+           o.min_rebalance_interval_ops >= 1 && o.max_requests >= 1 && o.max_pages_per_request >= 1 &&
+           (uint64_t)o.max_requests * o.max_pages_per_request < (1ull << 32);
+}
+
+inline cudaStream_t S(void *s) { return reinterpret_cast<cudaStream_t>(s); }
+inline Launch L(const avmp_ctx *c, void *s) { return Launch{S(s), c->n_sms}; }
+inline int cu(cudaError_t e) { return e == cudaSuccess ? AVMP_OK : AVMP_ECUDA; }
+
+void fill_stats(const avmp_ctx *c, const DevState &d, avmp_stats *o)
+{
+    o->op_counter = d.op_counter; o->last_rebalance_op = d.last_rebalance_op; o->n_oom = d.n_oom;
+    o->n_capacity_error = d.n_capacity_error; o->n_rebalance = d.n_rebalance;
+    o->migrated_bytes = d.migrated_bytes; o->wasted_bytes = d.wasted_bytes;
+    o->relocated_blocks = d.relocated_blocks; o->relocated_bytes = d.relocated_bytes;
+    o->gap_bytes = d.gap_bytes;
+    for (int p = 0; p < 2; ++p) {
+        o->cap[p] = d.cap[p]; o->free_units[p] = d.n_free[p];
+        o->unit_bytes[p] = c->lay.unit_bytes[p]; o->vid_space[p] = c->lay.vid_space[p];
+    }
+    o->fsm_state = d.fsm; o->n_invalid = d.n_invalid;
+    o->pool_bytes_aligned = c->lay.pool_bytes_aligned;
+    o->error_code = d.error_code; o->error_count = d.error_count;
+}
+
+}  // namespace
+
+extern "C" {
+
+void avmp_default_options(avmp_options *o)
+{
+    if (!o) return;
+    o->threshold_low_ppm = 50000; o->threshold_high_ppm = 300000;
+    o->min_rebalance_interval_ops = 1000; o->migration_enabled = 1;
+    o->max_requests = 1024; o->max_pages_per_request = 4096;
+}
+
+int avmp_derive_layout(const avmp_model_spec *m, uint64_t pool_bytes, double split, avmp_layout *out)
+{
+    if (!m || !out) return AVMP_EINVAL;
+    if (!(split >= 0.0 && split <= 1.0) || m->page_tokens == 0) return AVMP_EINVAL;
+    avmp_layout l;
+    l.kv_row_bytes = (uint64_t)m->kv_heads * m->head_dim * m->kv_elem_bytes;
+    l.kv_layer_bytes = 2ull * m->page_tokens * l.kv_row_bytes;
+    l.ssm_state_bytes = (uint64_t)m->ssm_state_elems * m->ssm_elem_bytes;
+    l.ssm_conv_bytes = (uint64_t)m->ssm_conv_elems * m->ssm_elem_bytes;
+    l.unit_bytes[0] = ((uint64_t)m->n_attn_layers * l.kv_layer_bytes + 15u) & ~15ull;
+    l.unit_bytes[1] = (l.ssm_state_bytes + l.ssm_conv_bytes + 15u) & ~15ull;
+    if (l.unit_bytes[0] == 0 || l.unit_bytes[1] == 0) return AVMP_EINVAL;
+    l.pool_bytes_aligned = pool_bytes & ~127ull;
+    const uint64_t ppm = (uint64_t)llround(split * 1e6);
+    const uint64_t ssm_bytes = (uint64_t)(((unsigned __int128)l.pool_bytes_aligned * ppm) / 1000000u) & ~127ull;
+    l.cap0[0] = (l.pool_bytes_aligned - ssm_bytes) / l.unit_bytes[0];
+    l.cap0[1] = ssm_bytes / l.unit_bytes[1];
+    l.gap0 = l.pool_bytes_aligned - l.cap0[0] * l.unit_bytes[0] - l.cap0[1] * l.unit_bytes[1];
+    for (int p = 0; p < 2; ++p) {
+        l.vid_space[p] = l.pool_bytes_aligned / l.unit_bytes[p];
+        if (l.vid_space[p] >= 0x7FFFFFFFull) return AVMP_EINVAL;
+    }
+    if (l.cap0[0] == 0 && l.cap0[1] == 0) return AVMP_EINVAL;
+    *out = l;
+    return AVMP_OK;
+}
+
+size_t avmp_workspace_bytes(const avmp_model_spec *spec, uint64_t pool_bytes, const avmp_options *opt)
+{
+    avmp_options o;
+    if (opt) o = *opt; else avmp_default_options(&o);
+    avmp_layout lay;
+    if (!spec || !options_ok(o) || avmp_derive_layout(spec, pool_bytes, 0.5, &lay) != AVMP_OK) return 0;
+    return ws_layout(lay, *spec, o).total;
+}
+
+int avmp_create(avmp_ctx **out, const avmp_model_spec *spec, void *d_arena, uint64_t pool_bytes,
+                double initial_split, uint32_t migration_batch_size, const avmp_options *opt,
+                void *d_workspace, size_t workspace_bytes, void *stream)
+{
+    if (!out || !spec || !d_arena || !d_workspace) return AVMP_EINVAL;
+    if (((uintptr_t)d_arena | (uintptr_t)d_workspace) & (kAlign - 1)) return AVMP_EINVAL;
+    avmp_options o;
+    if (opt) o = *opt; else avmp_default_options(&o);
+    if (!options_ok(o)) return AVMP_EINVAL;                       // Section 4.6: low >= high is invalid
+    avmp_layout lay;
+    if (avmp_derive_layout(spec, pool_bytes, initial_split, &lay) != AVMP_OK) return AVMP_EINVAL;
+    const WsLayout w = ws_layout(lay, *spec, o);
+    if (workspace_bytes < w.total) return AVMP_ENOSPC;
+
+    avmp_ctx *c = new (std::nothrow) avmp_ctx();
+    if (!c) return AVMP_EINVAL;
+    c->spec = *spec; c->opt = o; c->lay = lay; c->B = migration_batch_size; c->launches = 0;
+    c->d_workspace = d_workspace; c->workspace_bytes = workspace_bytes;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+        delete c;
+        return AVMP_ECUDA;
+    }
+    uint8_t *base = static_cast<uint8_t *>(d_workspace);
+    Geom &g = c->g;
+    g.P_al = lay.pool_bytes_aligned; g.U[0] = lay.unit_bytes[0]; g.U[1] = lay.unit_bytes[1];
+    g.kv_layer_bytes = lay.kv_layer_bytes; g.row_bytes = lay.kv_row_bytes;
+    g.state_bytes = lay.ssm_state_bytes; g.conv_bytes = lay.ssm_conv_bytes;
+    g.min_interval = o.min_rebalance_interval_ops;
+    g.V[0] = (uint32_t)lay.vid_space[0]; g.V[1] = (uint32_t)lay.vid_space[1];
+    g.T = spec->page_tokens; g.na = spec->n_attn_layers; g.ns = spec->n_ssm_layers;
+    g.R = o.max_requests; g.max_pages = o.max_pages_per_request; g.B = migration_batch_size;
+    g.th_low = o.threshold_low_ppm; g.th_high = o.threshold_high_ppm; g.migration_enabled = o.migration_enabled;
+    g.arena = static_cast<uint8_t *>(d_arena);
+    g.st = reinterpret_cast<DevState *>(base + w.state);
+    for (int p = 0; p < 2; ++p) {
+        g.S[p] = reinterpret_cast<uint32_t *>(base + w.S[p]); g.W[p] = reinterpret_cast<uint32_t *>(base + w.W[p]);
+        g.VT[p] = reinterpret_cast<uint32_t *>(base + w.VT[p]); g.OW[p] = reinterpret_cast<uint32_t *>(base + w.OW[p]);
+    }
+    g.r_state = reinterpret_cast<uint32_t *>(base + w.r_state); g.r_len = reinterpret_cast<uint32_t *>(base + w.r_len);
+    g.r_npages = reinterpret_cast<uint32_t *>(base + w.r_npages); g.r_chain = reinterpret_cast<uint32_t *>(base + w.r_chain);
+    g.r_ssm = reinterpret_cast<uint32_t *>(base + w.r_ssm); g.mark = reinterpret_cast<uint32_t *>(base + w.mark);
+    g.reloc_src = reinterpret_cast<uint32_t *>(base + w.reloc_src); g.reloc_dst = reinterpret_cast<uint32_t *>(base + w.reloc_dst);
+    g.g_cu_items = reinterpret_cast<uint32_t *>(base + w.g_cu_items); g.g_cu_rows = reinterpret_cast<uint32_t *>(base + w.g_cu_rows);
+    c->d_stage_ops = reinterpret_cast<avmp_op *>(base + w.stage_ops);
+    c->d_stage_status = reinterpret_cast<uint32_t *>(base + w.stage_status);
+
+    DevState init;
+    memset(&init, 0, sizeof(init));
+    init.last_rebalance_op = kNone64;
+    init.gap_bytes = lay.gap0;
+    for (int p = 0; p < 2; ++p) {
+        init.cap[p] = init.n_free[p] = (uint32_t)lay.cap0[p];
+        init.n_vfree[p] = (uint32_t)lay.vid_space[p];
+    }
+    init.fsm = AVMP_FSM_BALANCED;
+    if (launch_init(g, init, S(stream)) != cudaSuccess) { delete c; return AVMP_ECUDA; }
+    c->launches += 1;
+    *out = c;
+    return AVMP_OK;
+}
+
+int avmp_destroy(avmp_ctx *c)
+{
+    delete c;
+    return AVMP_OK;
+}
+
+int avmp_step(avmp_ctx *c, const avmp_op *d_ops, uint32_t n_ops, uint32_t *d_status, void *stream)
+{
+    if (!c) return AVMP_EINVAL;
+    if (n_ops == 0) return AVMP_OK;
+    if (!d_ops || !d_status || ((uintptr_t)d_ops & 3) || ((uintptr_t)d_status & 3)) return AVMP_EINVAL;
+    // Section 3.2 throttle: migrations are >= min_interval logical ops apart, so a batch of n ops
+    // holds at most (n - 1) / min_interval + 1 of them; one launch performs at most one.
+    uint32_t rounds = 1;
+    if (c->opt.migration_enabled)
+        rounds = (uint32_t)((n_ops - 1) / c->opt.min_rebalance_interval_ops) + 1;
+    for (uint32_t r = 0; r < rounds; ++r) {
+        if (launch_step(c->g, d_ops, n_ops, d_status, r == 0, S(stream)) != cudaSuccess) return AVMP_ECUDA;
+        c->launches += 1;
+        if (c->opt.migration_enabled) {
+            if (launch_relocate(c->g, L(c, stream)) != cudaSuccess) return AVMP_ECUDA;
+            c->launches += 1;
+        }
+    }
+    return AVMP_OK;
+}
+
+int avmp_step_host(avmp_ctx *c, const avmp_op *h_ops, uint32_t n_ops, uint32_t *h_status, void *stream)
+{
+    if (!c) return AVMP_EINVAL;
+    if (n_ops == 0) return AVMP_OK;
+    if (!h_ops || !h_status || n_ops > kHostStepMaxOps) return AVMP_EINVAL;
+    if (cudaMemcpyAsync(c->d_stage_ops, h_ops, (size_t)n_ops * sizeof(avmp_op), cudaMemcpyHostToDevice, S(stream)) != cudaSuccess)
+        return AVMP_ECUDA;
+    int rc = avmp_step(c, c->d_stage_ops, n_ops, c->d_stage_status, stream);
+    if (rc != AVMP_OK) return rc;
+    if (cudaMemcpyAsync(h_status, c->d_stage_status, (size_t)n_ops * 4, cudaMemcpyDeviceToHost, S(stream)) != cudaSuccess)
+        return AVMP_ECUDA;
+    return cu(cudaStreamSynchronize(S(stream)));
+}
+
+int avmp_translate(avmp_ctx *c, const uint32_t *d_handles, uint32_t n, uint32_t *d_pool,
+                   uint64_t *d_offset, uint64_t *d_arena_offset, void *stream)
+{
+    if (!c) return AVMP_EINVAL;
+    if (n == 0) return AVMP_OK;
+    if (!d_handles || !d_pool || !d_offset) return AVMP_EINVAL;
+    c->launches += 1;
+    return cu(launch_translate(c->g, d_handles, n, d_pool, (unsigned long long *)d_offset,
+                               (unsigned long long *)d_arena_offset, L(c, stream)));
+}
+
+int avmp_gather_kv(avmp_ctx *c, uint32_t layer, const uint32_t *d_reqs, uint32_t n, void *d_out_k,
+                   void *d_out_v, uint64_t cap_tokens, uint32_t *d_cu, void *stream)
+{
+    if (!c || layer >= c->spec.n_attn_layers || n > c->opt.max_requests || !d_cu) return AVMP_EINVAL;
+    if (n && (!d_reqs || !d_out_k || !d_out_v)) return AVMP_EINVAL;
+    if (((uintptr_t)d_out_k | (uintptr_t)d_out_v) & 15) return AVMP_EINVAL;
+    c->launches += 2;
+    return cu(launch_kv(c->g, false, layer, d_reqs, nullptr, n, d_out_k, d_out_v, cap_tokens, d_cu, L(c, stream)));
+}
+
+int avmp_scatter_kv(avmp_ctx *c, uint32_t layer, const uint32_t *d_reqs, const uint32_t *d_tok_start,
+                    uint32_t n, const void *d_in_k, const void *d_in_v, void *stream)
+{
+    if (!c || layer >= c->spec.n_attn_layers || n > c->opt.max_requests) return AVMP_EINVAL;
+    if (n == 0) return AVMP_OK;
+    if (!d_reqs || !d_in_k || !d_in_v || (((uintptr_t)d_in_k | (uintptr_t)d_in_v) & 15)) return AVMP_EINVAL;
+    c->launches += 2;
+    return cu(launch_kv(c->g, true, layer, d_reqs, d_tok_start, n, const_cast<void *>(d_in_k),
+                        const_cast<void *>(d_in_v), ~0ull, nullptr, L(c, stream)));
+}
+
+int avmp_gather_ssm(avmp_ctx *c, uint32_t layer, const uint32_t *d_reqs, uint32_t n, void *d_out_state,
+                    void *d_out_conv, void *stream)
+{
+    if (!c || layer >= c->spec.n_ssm_layers) return AVMP_EINVAL;
+    if (n == 0) return AVMP_OK;
+    if (!d_reqs || !d_out_state || !d_out_conv || (((uintptr_t)d_out_state | (uintptr_t)d_out_conv) & 15)) return AVMP_EINVAL;
+    c->launches += 1;
+    return cu(launch_ssm(c->g, false, layer, d_reqs, n, d_out_state, d_out_conv, L(c, stream)));
+}
+
+int avmp_scatter_ssm(avmp_ctx *c, uint32_t layer, const uint32_t *d_reqs, uint32_t n, const void *d_in_state,
+                     const void *d_in_conv, void *stream)
+{
+    if (!c || layer >= c->spec.n_ssm_layers) return AVMP_EINVAL;
+    if (n == 0) return AVMP_OK;
+    if (!d_reqs || !d_in_state || !d_in_conv || (((uintptr_t)d_in_state | (uintptr_t)d_in_conv) & 15)) return AVMP_EINVAL;
+    c->launches += 1;
+    return cu(launch_ssm(c->g, true, layer, d_reqs, n, const_cast<void *>(d_in_state),
+                         const_cast<void *>(d_in_conv), L(c, stream)));
+}
+
+int avmp_get_stats(avmp_ctx *c, avmp_stats *h_out, void *stream)
+{
+    if (!c || !h_out) return AVMP_EINVAL;
+    DevState d;
+    if (cudaMemcpyAsync(&d, c->g.st, sizeof(d), cudaMemcpyDeviceToHost, S(stream)) != cudaSuccess) return AVMP_ECUDA;
+    if (cudaStreamSynchronize(S(stream)) != cudaSuccess) return AVMP_ECUDA;
+    fill_stats(c, d, h_out);
+    return AVMP_OK;
+}
+
+int avmp_clear_error(avmp_ctx *c, void *stream)
+{
+    if (!c) return AVMP_EINVAL;
+    return cu(cudaMemsetAsync(&c->g.st->error_code, 0, 16, S(stream)));
+}
+
+int avmp_export_tables(avmp_ctx *c, avmp_tables *t, void *stream)
+{
+    if (!c || !t) return AVMP_EINVAL;
+    const Geom &g = c->g;
+    cudaStream_t s = S(stream);
+    DevState d;
+    bool ok = cudaMemcpyAsync(&d, g.st, sizeof(d), cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    auto pull = [&](uint32_t *dst, const uint32_t *src, size_t n) {
+        if (dst && n) ok = ok && cudaMemcpyAsync(dst, src, n * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    };
+    for (int p = 0; p < 2; ++p) {
+        pull(t->slot_stack[p], g.S[p], g.V[p]); pull(t->vid_stack[p], g.W[p], g.V[p]);
+        pull(t->vt[p], g.VT[p], g.V[p]); pull(t->ow[p], g.OW[p], g.V[p]);
+    }
+    pull(t->req_state, g.r_state, g.R); pull(t->req_len, g.r_len, g.R); pull(t->req_npages, g.r_npages, g.R);
+    pull(t->req_chain, g.r_chain, (size_t)g.R * g.max_pages); pull(t->req_ssm, g.r_ssm, (size_t)g.R * g.ns);
+    if (!ok || cudaStreamSynchronize(s) != cudaSuccess) return AVMP_ECUDA;
+    for (int p = 0; p < 2; ++p) { t->n_slot_stack[p] = d.n_free[p]; t->n_vid_stack[p] = d.n_vfree[p]; }
+    fill_stats(c, d, &t->stats);
+    return AVMP_OK;
+}
+
+int avmp_import_tables(avmp_ctx *c, const avmp_tables *t, void *stream)
+{
+    if (!c || !t) return AVMP_EINVAL;
+    const Geom &g = c->g;
+    cudaStream_t s = S(stream);
+    for (int p = 0; p < 2; ++p) {
+        if (!t->slot_stack[p] || !t->vid_stack[p] || !t->vt[p] || !t->ow[p]) return AVMP_EINVAL;
+        if (t->n_slot_stack[p] > g.V[p] || t->n_vid_stack[p] > g.V[p] || t->stats.cap[p] > g.V[p]) return AVMP_EINVAL;
+    }
+    if (!t->req_state || !t->req_len || !t->req_npages || !t->req_chain || (g.ns && !t->req_ssm)) return AVMP_EINVAL;
+    bool ok = true;
+    auto push = [&](uint32_t *dst, const uint32_t *src, size_t n) {
+        if (n) ok = ok && cudaMemcpyAsync(dst, src, n * 4, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    };
+    for (int p = 0; p < 2; ++p) {
+        push(g.S[p], t->slot_stack[p], g.V[p]); push(g.W[p], t->vid_stack[p], g.V[p]);
+        push(g.VT[p], t->vt[p], g.V[p]); push(g.OW[p], t->ow[p], g.V[p]);
+    }
+    push(g.r_state, t->req_state, g.R); push(g.r_len, t->req_len, g.R); push(g.r_npages, t->req_npages, g.R);
+    push(g.r_chain, t->req_chain, (size_t)g.R * g.max_pages); push(g.r_ssm, t->req_ssm, (size_t)g.R * g.ns);
+    DevState d;
+    memset(&d, 0, sizeof(d));
+    const avmp_stats &st = t->stats;
+    d.op_counter = st.op_counter; d.last_rebalance_op = st.last_rebalance_op; d.n_oom = st.n_oom;
+    d.n_capacity_error = st.n_capacity_error; d.n_rebalance = st.n_rebalance;
+    d.migrated_bytes = st.migrated_bytes; d.wasted_bytes = st.wasted_bytes;
+    d.relocated_blocks = st.relocated_blocks; d.relocated_bytes = st.relocated_bytes;
+    d.gap_bytes = st.gap_bytes; d.n_invalid = st.n_invalid;
+    for (int p = 0; p < 2; ++p) {
+        d.cap[p] = (uint32_t)st.cap[p]; d.n_free[p] = t->n_slot_stack[p]; d.n_vfree[p] = t->n_vid_stack[p];
+    }
+    d.fsm = (uint32_t)st.fsm_state;
+    ok = ok && cudaMemcpyAsync(g.st, &d, sizeof(d), cudaMemcpyHostToDevice, s) == cudaSuccess;
+    // the host arrays (and `d`) must outlive the copies
+    if (!ok || cudaStreamSynchronize(s) != cudaSuccess) return AVMP_ECUDA;
+    return AVMP_OK;
+}
+
+uint64_t avmp_launch_count(const avmp_ctx *c) { return c ? c->launches : 0; }
+
+const char *avmp_error_string(int code)
+{
+    switch (code) {
+    case AVMP_OK: return "ok";
+    case AVMP_EINVAL: return "invalid argument";
+    case AVMP_ENOSPC: return "workspace too small";
+    case AVMP_ECUDA: return "CUDA runtime error";
+    default: return "unknown error";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,128 @@
+// Device-side state, geometry and small block/warp primitives shared by the AVMP kernels.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "avmp.h"
+
+namespace avmp {
+
+constexpr uint32_t kInvalid = 0xFFFFFFFFu;
+constexpr unsigned long long kNone64 = 0xFFFFFFFFFFFFFFFFull;
+constexpr int kStepThreads = 1024;          // one CTA plans a step; one op per thread per window
+constexpr uint32_t kHostStepMaxOps = 65536; // staging capacity of avmp_step_host
+
+// Mutable allocator state, resident in the workspace (one instance per context).
+struct DevState {
+    unsigned long long op_counter, last_rebalance_op, n_oom, n_capacity_error, n_rebalance;
+    unsigned long long migrated_bytes, wasted_bytes, relocated_blocks, relocated_bytes, gap_bytes;
+    unsigned long long n_invalid, error_code, error_count;
+    uint32_t cap[2], n_free[2], n_vfree[2], fsm;
+    uint32_t resume_idx;     // ops of the batch in flight already applied (multi-round steps)
+    uint32_t n_reloc;        // relocation list of the last round
+    uint32_t reloc_pool;
+    uint32_t g_total_items;  // work items of the gather / scatter being planned
+    uint32_t pad;
+};
+
+// Immutable geometry + table pointers, passed to kernels by value.
+struct Geom {
+    unsigned long long P_al, U[2], kv_layer_bytes, row_bytes, state_bytes, conv_bytes, min_interval;
+    uint32_t V[2];
+    uint32_t T, na, ns, R, max_pages, B, th_low, th_high, migration_enabled;
+    uint8_t *arena;
+    DevState *st;
+    uint32_t *S[2], *W[2], *VT[2], *OW[2];
+    uint32_t *r_state, *r_len, *r_npages, *r_chain, *r_ssm, *mark;
+    uint32_t *reloc_src, *reloc_dst;
+    uint32_t *g_cu_items, *g_cu_rows;   // gather scratch, R + 1 entries each
+};
+
+// Byte address of a unit: KV slots grow up from the arena base, SSM slots grow down
+// from its end, so both stores shrink and grow at the gap between them.
+__device__ __forceinline__ uint8_t *unit_ptr(const Geom &g, uint32_t pool, uint32_t slot)
+{
+    return pool == AVMP_POOL_KV ? g.arena + (unsigned long long)slot * g.U[0]
+                                : g.arena + (g.P_al - ((unsigned long long)slot + 1ull) * g.U[1]);
+}
+
+__device__ __forceinline__ void record_error(DevState *st, unsigned long long code)
+{
+    atomicCAS(&st->error_code, 0ull, code);
+    atomicAdd(&st->error_count, 1ull);
+}
+
+// ---- warp / block primitives (blockDim.x == kStepThreads for the block ones) ----
+__device__ __forceinline__ unsigned long long warp_incl_scan(unsigned long long v)
+{
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        unsigned long long n = __shfl_up_sync(0xFFFFFFFFu, v, o);
+        if (lane >= o) v += n;
+    }
+    return v;
+}
+
+// Inclusive scan over the whole block; *total receives the block sum.  `tmp` is 32
+// words of shared memory; the call ends with a barrier so `tmp` can be reused at once.
+__device__ __forceinline__ unsigned long long block_incl_scan(unsigned long long v, unsigned long long *tmp,
+                                                              unsigned long long *total)
+{
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    v = warp_incl_scan(v);
+    if (lane == 31) tmp[wid] = v;
+    __syncthreads();
+    if (wid == 0) {
+        unsigned long long w = (lane < (int)(blockDim.x >> 5)) ? tmp[lane] : 0ull;
+        tmp[lane] = warp_incl_scan(w);
+    }
+    __syncthreads();
+    const unsigned long long off = wid ? tmp[wid - 1] : 0ull;
+    *total = tmp[31];
+    __syncthreads();
+    return v + off;
+}
+
+__device__ __forceinline__ uint32_t block_min(uint32_t v, uint32_t *tmp)
+{
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    v = __reduce_min_sync(0xFFFFFFFFu, v);
+    if (lane == 0) tmp[wid] = v;
+    __syncthreads();
+    uint32_t w = (lane < (int)(blockDim.x >> 5)) ? tmp[lane] : 0xFFFFFFFFu;
+    w = __reduce_min_sync(0xFFFFFFFFu, w);
+    __syncthreads();
+    return w;
+}
+
+// Largest idx in [lo, hi) with a[idx] - base <= u   (a is non-decreasing, a[lo] - base <= u).
+__device__ __forceinline__ uint32_t find_owner(const uint32_t *a, uint32_t lo, uint32_t hi, uint32_t base,
+                                               uint32_t u)
+{
+    while (lo + 1 < hi) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (a[mid] - base <= u) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// Host-side launch wrappers (defined next to their kernels).
+struct Launch {
+    cudaStream_t stream;
+    int n_sms;
+};
+cudaError_t launch_init(const Geom &g, const DevState &init, cudaStream_t s);
+cudaError_t launch_step(const Geom &g, const avmp_op *d_ops, uint32_t n_ops, uint32_t *d_status,
+                        int first_round, cudaStream_t s);
+cudaError_t launch_relocate(const Geom &g, const Launch &l);
+cudaError_t launch_translate(const Geom &g, const uint32_t *h, uint32_t n, uint32_t *pool,
+                             unsigned long long *off, unsigned long long *aoff, const Launch &l);
+cudaError_t launch_kv(const Geom &g, bool scatter, uint32_t layer, const uint32_t *reqs,
+                      const uint32_t *tok_start, uint32_t n, void *k, void *v,
+                      unsigned long long cap_tokens, uint32_t *cu_out, const Launch &l);
+cudaError_t launch_ssm(const Geom &g, bool scatter, uint32_t layer, const uint32_t *reqs, uint32_t n,
+                       void *state, void *conv, const Launch &l);
+
+}  // namespace avmp

@@ -1,0 +1,120 @@
+"""numpy-in / numpy-out adapter around the CUDA binding, with the same method names as the
+oracle wrapper, so the same test harness can drive both.  Test code only: it moves arrays
+to and from the device and calls the C ABI; it computes nothing."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from paper_2605_22416_b200 import binding as B
+
+
+class GpuEngine:
+    def __init__(self, w, device="cuda:0", **over):
+        self.w = w
+        self.dev = torch.device(device)
+        self.ctx = B.Context.from_workload(w, device=device, **over)
+        self.model = w.model
+        self.max_pages = self.ctx.opt.max_pages_per_request
+
+    def close(self):
+        self.ctx.close()
+
+    def _dev(self, a: np.ndarray, dtype=None) -> torch.Tensor:
+        a = np.ascontiguousarray(a if dtype is None else np.asarray(a, dtype=dtype))
+        if a.size == 0:
+            return torch.zeros(16, dtype=torch.uint8, device=self.dev)
+        return torch.from_numpy(a.view(np.uint8).reshape(-1)).to(self.dev)
+
+    def step(self, ops: np.ndarray) -> np.ndarray:
+        n = len(ops)
+        if n == 0:
+            self.ctx.step(0, 0, 0)
+            return np.zeros(0, np.uint32)
+        d_ops = self._dev(ops)
+        d_st = torch.full((n,), 0xEE, dtype=torch.int32, device=self.dev)
+        self.ctx.step(d_ops, n, d_st)
+        return d_st.cpu().numpy().view(np.uint32)
+
+    def step_host(self, ops: np.ndarray) -> np.ndarray:
+        ops = np.ascontiguousarray(ops)
+        st = np.full(len(ops), 0xEE, np.uint32)
+        self.ctx.step_host(ops, len(ops), st)
+        return st
+
+    def translate(self, handles):
+        h = np.ascontiguousarray(handles, dtype=np.uint32)
+        n = len(h)
+        d_h = self._dev(h)
+        pool = torch.zeros(max(n, 1), dtype=torch.int32, device=self.dev)
+        off = torch.zeros(max(n, 1), dtype=torch.int64, device=self.dev)
+        aoff = torch.zeros(max(n, 1), dtype=torch.int64, device=self.dev)
+        before = self.ctx.stats()["error_count"]
+        self.ctx.translate(d_h, n, pool, off, aoff)
+        bad = self.ctx.stats()["error_count"] - before
+        return (pool.cpu().numpy().view(np.uint32)[:n], off.cpu().numpy().view(np.uint64)[:n], bad,
+                aoff.cpu().numpy().view(np.uint64)[:n])
+
+    def gather_kv(self, layer, reqs, capacity_tokens):
+        r = np.ascontiguousarray(reqs, dtype=np.uint32)
+        row = self.model.kv_row_bytes
+        out_k = torch.zeros((max(capacity_tokens, 1), row), dtype=torch.uint8, device=self.dev)
+        out_v = torch.zeros((max(capacity_tokens, 1), row), dtype=torch.uint8, device=self.dev)
+        cu = torch.zeros(len(r) + 1, dtype=torch.int32, device=self.dev)
+        before = self.ctx.stats()["error_count"]
+        self.ctx.gather_kv(layer, self._dev(r), len(r), out_k, out_v, capacity_tokens, cu)
+        bad = self.ctx.stats()["error_count"] - before
+        return (out_k.cpu().numpy()[:capacity_tokens], out_v.cpu().numpy()[:capacity_tokens],
+                cu.cpu().numpy().view(np.uint32), bad)
+
+    def gather_ssm(self, layer, reqs):
+        r = np.ascontiguousarray(reqs, dtype=np.uint32)
+        n = len(r)
+        st = torch.zeros((max(n, 1), self.model.state_bytes), dtype=torch.uint8, device=self.dev)
+        cv = torch.zeros((max(n, 1), self.model.conv_bytes), dtype=torch.uint8, device=self.dev)
+        before = self.ctx.stats()["error_count"]
+        self.ctx.gather_ssm(layer, self._dev(r), n, st, cv)
+        bad = self.ctx.stats()["error_count"] - before
+        return st.cpu().numpy()[:n], cv.cpu().numpy()[:n], bad
+
+    def scatter_kv(self, layer, reqs, tok_start, in_k, in_v) -> int:
+        r = np.ascontiguousarray(reqs, dtype=np.uint32)
+        before = self.ctx.stats()["error_count"]
+        self.ctx.scatter_kv(layer, self._dev(r), self._dev(tok_start, np.uint32), len(r),
+                            self._dev(in_k), self._dev(in_v))
+        return self.ctx.stats()["error_count"] - before
+
+    def scatter_ssm(self, layer, reqs, in_state, in_conv) -> int:
+        r = np.ascontiguousarray(reqs, dtype=np.uint32)
+        before = self.ctx.stats()["error_count"]
+        self.ctx.scatter_ssm(layer, self._dev(r), len(r), self._dev(in_state), self._dev(in_conv))
+        return self.ctx.stats()["error_count"] - before
+
+    def stats(self) -> dict:
+        return self.ctx.stats()
+
+    def tables(self) -> dict:
+        return self.ctx.export_tables()[0]
+
+
+def comparable_tables(t: dict, max_requests: int, max_pages: int, n_ssm_layers: int) -> dict:
+    """Tables reduced to what is defined: chains up to n_pages, SSM handles of LIVE slots."""
+    out = {k: v for k, v in t.items() if not k.startswith("req_chain") and not k.startswith("req_ssm")}
+    npg = t["req_npages"]
+    chain = t["req_chain"].reshape(max_requests, max_pages)
+    mask = np.arange(max_pages)[None, :] < npg[:, None]
+    out["req_chain"] = np.where(mask, chain, 0)
+    if n_ssm_layers:
+        ssm = t["req_ssm"].reshape(max_requests, n_ssm_layers)
+        out["req_ssm"] = np.where((t["req_state"] == 1)[:, None], ssm, 0)
+    return out
+
+
+def assert_same_state(gpu, oracle, w, what=""):
+    gs, os_ = gpu.stats(), oracle.stats()
+    for k, v in os_.items():
+        assert gs[k] == v, f"{what}: stat {k}: gpu {gs[k]} != oracle {v}"
+    gt = comparable_tables(gpu.tables(), gpu.ctx.opt.max_requests, gpu.max_pages, w.model.n_ssm_layers)
+    ot = comparable_tables(oracle.tables(), oracle.max_requests, oracle.max_pages, w.model.n_ssm_layers)
+    for k in ot:
+        assert np.array_equal(gt[k], ot[k]), f"{what}: table {k} differs"

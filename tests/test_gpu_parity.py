@@ -1,0 +1,306 @@
+"""GPU parity: the CUDA path through the C ABI against the CPU oracle, bit for bit
+(tolerance 0: the path performs no floating-point arithmetic)."""
+from __future__ import annotations
+
+from pathlib import Path
+
+import numpy as np
+import pytest
+
+from harness import PayloadHarness
+from invariants import check_invariants
+from paper_2605_22416_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+GOLDEN = Path(__file__).resolve().parent / "golden"
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    from gpu_engine import GpuEngine, assert_same_state
+    from oracle.avmp_oracle import Oracle
+    assert torch.cuda.is_available()
+    return dict(GpuEngine=GpuEngine, Oracle=Oracle, same=assert_same_state, torch=torch)
+
+
+def _pair(env, w, with_store=False, **over):
+    g = env["GpuEngine"](w, **over)
+    o = env["Oracle"].from_workload(w, with_store=with_store, **over)
+    return g, o
+
+
+def test_library_is_loaded_from_the_tree(env):
+    from paper_2605_22416_b200 import binding
+    assert Path(binding.LIBRARY_PATH).exists()
+    maps = Path("/proc/self/maps").read_text()
+    assert "libavmp.so" in maps
+
+
+def test_worked_example_on_gpu(env):
+    w = W.config("tiny")
+    g = env["GpuEngine"](w)
+    kinds = {"ADMIT": 1, "EXTEND": 2, "FINISH": 3}
+    cols = ("cap_kv", "free_kv", "cap_ssm", "free_ssm", "gap_bytes", "migrated_bytes", "wasted_bytes",
+            "n_rebalance", "relocated_blocks", "n_oom", "n_capacity_error")
+    for line in (GOLDEN / "worked_example.txt").read_text().splitlines():
+        if "|" not in line or line.startswith("#"):
+            continue
+        l, r = line.split("|")
+        k, req, tok = l.split()
+        exp = [int(x) for x in r.split()]
+        st = g.step(W.make_ops(kinds[k], [int(req)], int(tok)))
+        s = g.stats()
+        assert int(st[0]) == exp[0], line
+        assert [s[c] for c in cols] == exp[1:12], line
+    pool, off, bad, aoff = g.translate(np.array([9, 8, 2, (1 << 31) | 2], np.uint32))
+    assert bad == 0 and pool.tolist() == [0, 0, 0, 1] and off.tolist() == [128, 512, 64, 192]
+    # arena placement: KV grows up from 0, SSM slot j ends at pool_end - j * U
+    assert aoff.tolist() == [128, 512, 64, 1024 - 3 * 96]
+
+
+@pytest.mark.parametrize("seed,batch", [(0, 1), (1, 7), (2, 32), (3, 300), (4, 1500)])
+def test_random_op_strings_tiny(env, seed, batch):
+    """Unscheduled ops (any order, repeated slots inside a batch, invalid ops): statuses,
+    counters and every table equal the oracle's after each batch."""
+    w = W.config("tiny", migration_batch_size=1 + seed % 4)
+    g, o = _pair(env, w, max_requests=6, max_pages=8)
+    ops = W.random_op_string(100 + seed, 3000, 6, 60)
+    for i in range(0, len(ops), batch):
+        b = ops[i:i + batch]
+        sg, so = g.step(b), o.step(b)
+        assert np.array_equal(sg, so), (i, sg[:20], so[:20])
+        if (i // batch) % 5 == 0 or batch >= 300:
+            env["same"](g, o, w, f"batch at {i}")
+    env["same"](g, o, w, "end")
+    s = g.stats()
+    assert s["n_rebalance"] > 0 and s["relocated_blocks"] > 0 and s["n_oom"] > 0
+    check_invariants(s, g.tables(), page_tokens=16, n_ssm_layers=1, max_pages=8)
+
+
+def test_many_migrations_inside_one_batch(env):
+    """min_interval 1: a single batch holds many migrations in both directions, so the step
+    runs as several plan/copy rounds; payload must follow every relocation."""
+    w = W.config("tiny", migration_batch_size=2, min_rebalance_interval_ops=1, pool_bytes=4096)
+    g, o = _pair(env, w, with_store=True, max_requests=16, max_pages=8)
+    rng = np.random.default_rng(3)
+    for rnd in range(30):
+        ops = W.random_op_string(500 + rnd, 64, 16, 90, p_invalid=0.02)
+        sg, so = g.step(ops), o.step(ops)
+        assert np.array_equal(sg, so)
+        env["same"](g, o, w, f"round {rnd}")
+        # write fresh bytes for every token / block both sides hold, then read them back
+        t = o.tables()
+        held = np.flatnonzero(t["req_state"] != 0).astype(np.uint32)
+        lens = t["req_len"][held]
+        tot = int(lens.sum())
+        kb = rng.integers(0, 256, (tot, 2), dtype=np.uint8)
+        vb = rng.integers(0, 256, (tot, 2), dtype=np.uint8)
+        zeros = np.zeros(len(held), np.uint32)
+        for e in (g, o):
+            assert e.scatter_kv(0, held, zeros, kb, vb) == 0
+        live = np.flatnonzero(t["req_state"] == 1).astype(np.uint32)
+        sb = rng.integers(0, 256, (len(live), 80), dtype=np.uint8)
+        cb = rng.integers(0, 256, (len(live), 16), dtype=np.uint8)
+        for e in (g, o):
+            assert e.scatter_ssm(0, live, sb, cb) == 0
+        # a batch of pure growth: forces migrations that relocate what was just written
+        grow = W.make_ops(W.OP_EXTEND, live, 17)
+        assert np.array_equal(g.step(grow), o.step(grow))
+        env["same"](g, o, w, f"round {rnd} after growth")
+        t = o.tables()
+        new_lens = t["req_len"][held]
+        tot = int(new_lens.sum())
+        gk, gv, gcu, gb = g.gather_kv(0, held, tot)
+        ok, ov, ocu, ob = o.gather_kv(0, held, tot)
+        assert gb == ob == 0 and np.array_equal(gcu, ocu)
+        # tokens appended by `grow` were never written: compare the written prefix of each request
+        src = np.concatenate([[0], np.cumsum(lens)])
+        for k in range(len(held)):
+            a0, n_old = int(gcu[k]), int(lens[k])
+            assert np.array_equal(gk[a0:a0 + n_old], kb[src[k]:src[k] + n_old])
+            assert np.array_equal(gv[a0:a0 + n_old], vb[src[k]:src[k] + n_old])
+            assert np.array_equal(ok[a0:a0 + n_old], kb[src[k]:src[k] + n_old])
+        gs, gc, gb = g.gather_ssm(0, live)
+        os_, oc, ob = o.gather_ssm(0, live)
+        assert gb == ob == 0 and np.array_equal(gs, sb) and np.array_equal(gc, cb)
+        assert np.array_equal(os_, sb) and np.array_equal(oc, cb)
+    assert g.stats()["n_rebalance"] > 20 and g.stats()["relocated_blocks"] > 5
+
+
+def _closed_loop_parity(env, w, steps, *, with_store, kv_layers, ssm_layers, table_every, gather_every,
+                        oracle_store_checks=True):
+    g, o = _pair(env, w, with_store=with_store)
+    engines = [g, o] if with_store else [g]
+    h = PayloadHarness(w, engines, kv_layers=kv_layers, ssm_layers=ssm_layers)
+    seen = dict(reb=0, tokens=0)
+
+    def step(ops):
+        so = o.step(ops)
+        sg = g.step(ops)
+        assert np.array_equal(sg, so), f"statuses differ at step {d.step}"
+        return so
+
+    d = W.ClosedLoopDriver(w)
+
+    def on_step(d, ops, status):
+        h.apply_writes(d.writes)
+        s = o.stats()
+        migrated = s["n_rebalance"] != seen["reb"]
+        seen["reb"] = s["n_rebalance"]
+        if d.step % table_every == 0 or migrated:
+            env["same"](g, o, w, f"step {d.step}")
+        if d.step % gather_every == 0 or migrated:
+            kl = kv_layers[d.step % len(kv_layers)]
+            sl = ssm_layers[d.step % len(ssm_layers)]
+            seen["tokens"] += h.check_gathers(d, kl, sl)
+            if with_store:
+                # the two implementations against each other, including translate of live handles
+                run = d.running_slots.astype(np.uint32)
+                t = o.tables()
+                handles = np.concatenate([t["req_chain"].reshape(w.max_requests, w.max_pages)[r, :t["req_npages"][r]]
+                                          for r in run] + [t["req_ssm"].reshape(w.max_requests, -1)[run].reshape(-1)])
+                pg, og, bg, _ = g.translate(handles)
+                po, oo, bo = o.translate(handles)
+                assert bg == bo == 0 and np.array_equal(pg, po) and np.array_equal(og, oo)
+
+    W.record_trace(w, step, max_steps=steps, driver=d, on_step=on_step)
+    env["same"](g, o, w, "end")
+    s = g.stats()
+    check_invariants(s, g.tables(), page_tokens=w.model.page_tokens, n_ssm_layers=w.model.n_ssm_layers,
+                     max_pages=w.max_pages)
+    assert s["error_code"] == 0
+    return s, seen, d
+
+
+def test_pr1_every_step(env):
+    """Config 1 in full: statuses every step, all tables and counters every step, full gathers
+    of the running batch (GPU == oracle == payload function) every few steps."""
+    w = W.config("pr1")
+    s, seen, d = _closed_loop_parity(env, w, None, with_store=True, kv_layers=[0, 3], ssm_layers=[0, 11],
+                                     table_every=1, gather_every=5)
+    assert d.completed == 2000 and s["n_rebalance"] > 10 and s["n_oom"] > 100
+    assert seen["tokens"] > 1_000_000
+
+
+def test_pr1_small_pool_relocations(env):
+    """Config 1's model in a pool small enough that migrations must move live blocks."""
+    w = W.config("pr1", pool_bytes=24 * W.MiB, concurrency=12, min_rebalance_interval_ops=50,
+                 migration_batch_size=6, n_requests=300)
+    s, seen, d = _closed_loop_parity(env, w, 1500, with_store=True, kv_layers=[1, 2], ssm_layers=[3, 7],
+                                     table_every=1, gather_every=3)
+    assert s["relocated_blocks"] > 10 and s["n_rebalance"] > 5
+
+
+@pytest.mark.parametrize("name,steps,over", [
+    ("short_uniform", 1200, {}),
+    ("short_uniform", 500, dict(seed=1)),
+    ("short_uniform", 500, dict(seed=2, migration_enabled=False)),
+    ("mixed_long", 1200, dict(migration_batch_size=4)),
+    ("mixed_long", 1200, dict(migration_batch_size=16)),
+    ("mixed_long", 1200, dict(migration_batch_size=64)),
+    ("mixed_long", 600, dict(migration_batch_size=16, split=0.1)),
+    ("agentic_burst", 2500, {}),
+])
+def test_full_size_configs(env, name, steps, over):
+    """Configs 2-4 at their full pool sizes and step batches: statuses and counters every
+    step, tables every 64 steps and after every migration, gathers of the running batch on
+    one attention and one SSM layer against the payload function."""
+    w = W.config(name, **over)
+    s, seen, d = _closed_loop_parity(env, w, steps, with_store=False, kv_layers=[1], ssm_layers=[5],
+                                     table_every=64, gather_every=97)
+    assert seen["tokens"] > 0
+    if w.migration_enabled:
+        assert s["n_rebalance"] > 0
+    if name == "agentic_burst":
+        assert s["relocated_blocks"] > 100
+
+
+@pytest.mark.parametrize("split,enabled", [(0.5, True), (0.5, False), (0.9, False)])
+def test_scale_config(env, split, enabled):
+    """Config 5: 72-layer model, 120 GiB pool resident in HBM, step batch 1024."""
+    w = W.config("scale", split=split, migration_enabled=enabled)
+    s, seen, d = _closed_loop_parity(env, w, 400, with_store=False, kv_layers=[4], ssm_layers=[31],
+                                     table_every=100, gather_every=133)
+    assert seen["tokens"] > 0 and s["op_counter"] > 200_000
+
+
+def test_edge_cases(env):
+    w = W.config("tiny")
+    g, o = _pair(env, w, with_store=True)
+    assert len(g.step(np.zeros(0, W.OP_DTYPE))) == 0                     # empty batch
+    ops = W.make_ops(W.OP_ADMIT, [0, 1], [20, 5])
+    assert np.array_equal(g.step(ops), o.step(ops))
+    fin = W.make_ops(W.OP_FINISH, [1], 0, W.FLAG_KEEP_KV)
+    assert np.array_equal(g.step(fin), o.step(fin))
+    # gather error items: empty slot, capacity overflow, KV_ONLY request in an SSM gather
+    for reqs, cap in (([0, 3, 1], 25), ([0, 1], 22), ([0, 1], 25), ([], 0)):
+        gk, gv, gcu, gb = g.gather_kv(0, reqs, cap)
+        ok, ov, ocu, ob = o.gather_kv(0, reqs, cap)
+        assert gb == ob and np.array_equal(gcu, ocu), (reqs, cap)
+    assert g.stats()["error_code"] in (2, 3) and g.stats()["error_count"] == 2
+    g.ctx.clear_error()
+    assert g.stats()["error_count"] == 0
+    gs, gc, gb = g.gather_ssm(0, [0, 1])
+    assert gb == 1 and g.stats()["error_code"] == 2
+    # translate: dead and out-of-range handles
+    hs = np.array([0, 1, 2, 0xFFFFFFFF, (1 << 31) | 0, (1 << 31) | 1, 500], np.uint32)
+    pg, og, bg, _ = g.translate(hs)
+    po, oo, bo = o.translate(hs)
+    assert bg == bo == 4 and np.array_equal(pg, po) and np.array_equal(og, oo)
+    # host-buffer entry point
+    ops = W.random_op_string(9, 200, 8, 40)
+    assert np.array_equal(g.step_host(ops), o.step(ops))
+    env["same"](g, o, w, "after step_host")
+
+
+def test_create_rejects_bad_configurations(env):
+    from paper_2605_22416_b200 import binding as B
+    torch = env["torch"]
+    spec = B.model_spec(W.TINY_MODEL)
+    arena = torch.empty(4096, dtype=torch.uint8, device="cuda")
+    opt = B.avmp_default_options()
+    opt.max_requests, opt.max_pages_per_request = 4, 4
+    ws_bytes = B.avmp_workspace_bytes(spec, 1024, opt)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    bad = B.avmp_options(300_000, 300_000, 1000, 1, 4, 4)        # threshold_low >= threshold_high
+    with pytest.raises(B.AvmpError):
+        B.avmp_create(spec, arena, 1024, 0.5, 1, bad, ws, ws_bytes)
+    with pytest.raises(B.AvmpError):
+        B.avmp_create(spec, arena, 1024, 0.5, 1, opt, ws, ws_bytes - 256)   # workspace too small
+    with pytest.raises(B.AvmpError):
+        B.avmp_create(spec, arena, 1024, 1.5, 1, opt, ws, ws_bytes)          # split outside [0, 1]
+    with pytest.raises(B.AvmpError):
+        B.avmp_create(spec, arena.data_ptr() + 8, 1024, 0.5, 1, opt, ws, ws_bytes)  # misaligned arena
+    h = B.avmp_create(spec, arena, 1024, 0.5, 1, opt, ws, ws_bytes)
+    B.avmp_destroy(h)
+
+
+def test_export_import_roundtrip(env):
+    """Snapshot / restore: tables built by the oracle drive the GPU gathers directly."""
+    w = W.config("pr1", pool_bytes=24 * W.MiB, concurrency=12, min_rebalance_interval_ops=50,
+                 migration_batch_size=6, n_requests=60)
+    g, o = _pair(env, w, with_store=True)
+    h = PayloadHarness(w, [g, o], kv_layers=[0], ssm_layers=[0])
+    d = W.ClosedLoopDriver(w)
+
+    def step(ops):
+        so = o.step(ops)
+        assert np.array_equal(g.step(ops), so)
+        return so
+
+    W.record_trace(w, step, max_steps=150, driver=d, on_step=lambda d, a, b: h.apply_writes(d.writes))
+    tables, stats = g.ctx.export_tables()
+    g2 = env["GpuEngine"](w, arena=g.ctx.arena)           # same payload bytes, fresh tables
+    g2.ctx.import_tables(o.tables(), o.stats())            # tables from the ORACLE
+    env["same"](g2, o, w, "imported")
+    assert h.check_gathers(d, 0, 0, engines=[g2]) > 0
+    # and the imported context keeps stepping identically
+    def step2(ops):
+        so = o.step(ops)
+        assert np.array_equal(g2.step(ops), so)
+        return so
+
+    W.record_trace(w, step2, max_steps=200, driver=d)
+    env["same"](g2, o, w, "after more steps")
