@@ -1,0 +1,449 @@
+#!/usr/bin/env python
+"""Benchmark of the AVMP hot path on B200.
+
+One "step" = one engine step of the whole path on one batch of the closed-loop trace:
+avmp_step (admit / extend / finish batch, CapacityError handler, migration + relocation
+copy), avmp_translate of every live handle of the running batch, avmp_gather_kv for every
+attention layer and avmp_gather_ssm for every SSM layer of the running batch.
+
+Workload: the short-uniform mix (Jamba-like 4 attention + 28 Mamba layers, 4 GiB pool,
+split 0.5, B = 128, step batch 256), synthetic and seeded.  The trace is produced closed
+loop against the library itself (untimed), then replayed from device-resident op batches
+for the timed region.  Inputs exceed L2: every step reads and writes several GB.
+
+Prints ONE JSON line (see README for the fields).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+from paper_2605_22416_b200 import workloads as W  # noqa: E402
+
+METRIC = "paged gather+migration GB/s over whole engine steps (allocator ops/s reported beside it)"
+WARM_STEPS = 600          # closed-loop steps before the measured window (steady state)
+# DRAM bytes (read + write) per launch of the dominant kernel divided by its algorithmic bytes,
+# from the ncu capture summarised in profiles/ssm_gather_short_uniform.md; None until measured.
+NCU_TRAFFIC_RATIO = None
+
+
+def _peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        return float(json.loads(p.read_text())["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# ---------------------------------------------------------------------------------------
+# clocks during the timed region (NVML, read-only)
+# ---------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._t = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                for bit, name in self.REASONS.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(0.02)
+
+    def start(self):
+        if self.nv is not None:
+            self._t = threading.Thread(target=self._run, daemon=True)
+            self._t.start()
+
+    def stop(self) -> dict:
+        self._stop.set()
+        if self._t is not None:
+            self._t.join()
+        med = int(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# ---------------------------------------------------------------------------------------
+# bytes moved by one step, by definition of the operations (not by counting kernel traffic)
+# ---------------------------------------------------------------------------------------
+def step_bytes(model: W.ModelShape, n_running: int, total_tokens: int, relocated_bytes: int) -> dict:
+    kv = 2 * total_tokens * 2 * model.kv_row_bytes * model.n_attn_layers          # K and V, read + write
+    ssm = 2 * n_running * (model.state_bytes + model.conv_bytes) * model.n_ssm_layers
+    return {"kv": kv, "ssm": ssm, "reloc": 2 * relocated_bytes}
+
+
+def reduce_over_ranks(local_ms: float, local_sums: np.ndarray, world: int):
+    """max of the time, sum of the additive quantities, over all ranks (identity at world 1)."""
+    if world == 1:
+        return local_ms, local_sums
+    import torch
+    import torch.distributed as dist
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([local_ms], dtype=torch.float64, device=dev)
+    s = torch.tensor(local_sums, dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(s, op=dist.ReduceOp.SUM)
+    return float(t.item()), s.cpu().numpy()
+
+
+# ---------------------------------------------------------------------------------------
+# our arm
+# ---------------------------------------------------------------------------------------
+def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
+    import torch
+    from paper_2605_22416_b200 import binding as B
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    w = W.config(args.workload, seed=rank % 3 if world > 1 else args.seed)
+    m = w.model
+    n_steps = WARM_STEPS + args.warmup + args.steps
+
+    # ---- phase A: closed loop against the library (untimed) -> per-step batches ----
+    ctx = B.Context.from_workload(w, device=dev)
+    drv = W.ClosedLoopDriver(w)
+    trace = []
+    while not drv.done and drv.step < n_steps:
+        ops = drv.next_batch()
+        st = np.zeros(len(ops), np.uint32)
+        ctx.step_host(np.ascontiguousarray(ops), len(ops), st)
+        drv.feed(st)
+        rec = {"ops": ops, "run": drv.running_slots.astype(np.uint32), "lens": drv.len[drv.running_slots].copy()}
+        if drv.step > WARM_STEPS:
+            t, _ = ctx.export_tables()
+            chain = t["req_chain"].reshape(w.max_requests, w.max_pages)
+            ssm = t["req_ssm"].reshape(w.max_requests, m.n_ssm_layers)
+            rec["handles"] = np.concatenate([chain[r, :t["req_npages"][r]] for r in rec["run"]] +
+                                            [ssm[rec["run"]].reshape(-1)]).astype(np.uint32)
+        trace.append(rec)
+    assert len(trace) == n_steps, "trace ended before the measured window"
+    stats_a = ctx.stats()
+    arena = ctx.arena
+    ctx.close()
+
+    # ---- phase B: replay from device-resident batches ----
+    ctx = B.Context.from_workload(w, device=dev, arena=arena)
+    stream = torch.cuda.current_stream()
+    max_run = max(len(r["run"]) for r in trace[WARM_STEPS:])
+    max_tok = max(int(r["lens"].sum()) for r in trace[WARM_STEPS:])
+    max_h = max(len(r["handles"]) for r in trace[WARM_STEPS:])
+    d_status = torch.zeros(w.concurrency * 2 + 16, dtype=torch.int32, device=dev)
+    out_k = [torch.empty((max_tok, m.kv_row_bytes), dtype=torch.uint8, device=dev) for _ in range(m.n_attn_layers)]
+    out_v = [torch.empty((max_tok, m.kv_row_bytes), dtype=torch.uint8, device=dev) for _ in range(m.n_attn_layers)]
+    out_s = [torch.empty((max_run, m.state_bytes), dtype=torch.uint8, device=dev) for _ in range(m.n_ssm_layers)]
+    out_c = [torch.empty((max_run, m.conv_bytes), dtype=torch.uint8, device=dev) for _ in range(m.n_ssm_layers)]
+    d_cu = torch.zeros(max_run + 1, dtype=torch.int32, device=dev)
+    d_pool = torch.zeros(max_h, dtype=torch.int32, device=dev)
+    d_off = torch.zeros(max_h, dtype=torch.int64, device=dev)
+    d_aoff = torch.zeros(max_h, dtype=torch.int64, device=dev)
+
+    def to_dev(a):
+        a = np.ascontiguousarray(a)
+        return torch.from_numpy(a.view(np.uint8).reshape(-1)).to(dev) if a.size else torch.zeros(16, dtype=torch.uint8, device=dev)
+
+    for r in trace:
+        r["d_ops"] = to_dev(r["ops"])
+    for r in trace[WARM_STEPS:]:
+        r["d_run"] = to_dev(r["run"])
+        r["d_handles"] = to_dev(r["handles"])
+
+    for r in trace[:WARM_STEPS]:
+        ctx.step(r["d_ops"], len(r["ops"]), d_status, stream)
+    torch.cuda.synchronize(dev)
+    reloc0 = ctx.stats()["relocated_bytes"]
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def full_step(r, marks=None):
+        n_ops, n_run = len(r["ops"]), len(r["run"])
+        cap_tok = int(r["lens"].sum())
+        if marks is not None:
+            marks.append(("step", ev(), ev()))
+            marks[-1][1].record(stream)
+        ctx.step(r["d_ops"], n_ops, d_status, stream)
+        ctx.translate(r["d_handles"], len(r["handles"]), d_pool, d_off, d_aoff, stream)
+        if marks is not None:
+            marks[-1][2].record(stream)
+        for l in range(m.n_attn_layers):
+            if marks is not None:
+                marks.append(("kv", ev(), ev()))
+                marks[-1][1].record(stream)
+            ctx.gather_kv(l, r["d_run"], n_run, out_k[l], out_v[l], cap_tok, d_cu, stream)
+            if marks is not None:
+                marks[-1][2].record(stream)
+        for l in range(m.n_ssm_layers):
+            if marks is not None:
+                marks.append(("ssm", ev(), ev()))
+                marks[-1][1].record(stream)
+            ctx.gather_ssm(l, r["d_run"], n_run, out_s[l], out_c[l], stream)
+            if marks is not None:
+                marks[-1][2].record(stream)
+
+    for r in trace[WARM_STEPS:WARM_STEPS + args.warmup]:
+        full_step(r)
+    timed = trace[WARM_STEPS + args.warmup:]
+
+    # ---- timed region 1: K whole steps, one pair of events, no per-kernel events inside ----
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize(dev)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = ctx.launch_count()
+    e0, e1 = ev(), ev()
+    e0.record(stream)
+    for r in timed:
+        full_step(r)
+    e1.record(stream)
+    torch.cuda.synchronize(dev)
+    if world > 1:
+        dist.barrier()
+    total_ms = e0.elapsed_time(e1)
+    launches = ctx.launch_count() - launches0
+    st_b = ctx.stats()
+    reloc_bytes = st_b["relocated_bytes"] - reloc0   # includes warm-up steps' relocations: subtract below
+
+    # ---- timed region 2 (same steps cannot be replayed: state moved on); per-kernel durations come
+    # from a second replay of the same window on a fresh context, with events around each call ----
+    ctx.close()
+    ctx = B.Context.from_workload(w, device=dev, arena=arena)
+    for r in trace[:WARM_STEPS]:
+        ctx.step(r["d_ops"], len(r["ops"]), d_status, stream)
+    for r in trace[WARM_STEPS:WARM_STEPS + args.warmup]:
+        full_step(r)
+    torch.cuda.synchronize(dev)
+    reloc_w = ctx.stats()["relocated_bytes"]
+    marks = []
+    for r in timed:
+        full_step(r, marks)
+    torch.cuda.synchronize(dev)
+    clocks = sampler.stop()
+    st_c = ctx.stats()
+    reloc_timed = st_c["relocated_bytes"] - reloc_w
+    per = {"step": [], "kv": [], "ssm": []}
+    for kind, a, b in marks:
+        per[kind].append(a.elapsed_time(b))
+
+    # ---- e2e: host buffers in, host results out, every step ----
+    ctx.close()
+    ctx = B.Context.from_workload(w, device=dev, arena=arena)
+    for r in trace[:WARM_STEPS + args.warmup]:
+        ctx.step(r["d_ops"], len(r["ops"]), d_status, stream)
+    torch.cuda.synchronize(dev)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.uint8).reshape(-1).copy()).pin_memory()
+    h_ops = [np.ascontiguousarray(r["ops"]) for r in timed]
+    h_run = [pin(r["run"]) for r in timed]
+    h_status = np.zeros(w.concurrency * 2 + 16, np.uint32)
+    h_cu = torch.zeros(max_run + 1, dtype=torch.int32).pin_memory()
+    d_run_buf = torch.zeros(max_run * 4 + 16, dtype=torch.uint8, device=dev)
+    h2d = d2h = 0
+    torch.cuda.synchronize(dev)
+    t0 = time.perf_counter()
+    for r, ho, hr in zip(timed, h_ops, h_run):
+        n_ops, n_run = len(r["ops"]), len(r["run"])
+        ctx.step_host(ho, n_ops, h_status, stream)                 # H2D ops, D2H statuses, sync
+        d_run_buf[: hr.numel()].copy_(hr, non_blocking=True)       # H2D running list
+        cap_tok = int(r["lens"].sum())
+        for l in range(m.n_attn_layers):
+            ctx.gather_kv(l, d_run_buf, n_run, out_k[l], out_v[l], cap_tok, d_cu, stream)
+        for l in range(m.n_ssm_layers):
+            ctx.gather_ssm(l, d_run_buf, n_run, out_s[l], out_c[l], stream)
+        h_cu[: n_run + 1].copy_(d_cu[: n_run + 1], non_blocking=True)   # D2H row offsets of the batch
+        torch.cuda.synchronize(dev)
+        h2d += n_ops * 12 + n_run * 4
+        d2h += n_ops * 4 + (n_run + 1) * 4
+    e2e_ms = (time.perf_counter() - t0) * 1e3
+    ctx.close()
+
+    # ---- accounting ----
+    K = len(timed)
+    by = [step_bytes(m, len(r["run"]), int(r["lens"].sum()), 0) for r in timed]
+    kv_bytes = sum(b["kv"] for b in by)
+    ssm_bytes = sum(b["ssm"] for b in by)
+    moved = kv_bytes + ssm_bytes + 2 * reloc_timed
+    n_ops_total = sum(len(r["ops"]) for r in timed)
+    local_sums = np.array([moved, n_ops_total, kv_bytes, ssm_bytes, launches, h2d, d2h], dtype=np.float64)
+    total_ms_g, sums = reduce_over_ranks(total_ms, local_sums, world)
+    e2e_ms_g, _ = reduce_over_ranks(e2e_ms, np.zeros(1), world)
+    peak, peak_kind = _peaks()
+
+    ssm_launch_bytes = ssm_bytes / (K * m.n_ssm_layers)
+    ssm_avg_ms = float(np.mean(per["ssm"]))
+    achieved = ssm_launch_bytes / (ssm_avg_ms * 1e-3) / 1e9
+    kv_avg_ms = float(np.mean(per["kv"]))
+    step_avg_ms = float(np.mean(per["step"]))
+    out = {
+        "metric": METRIC, "value": sums[0] / (total_ms_g * 1e-3) / 1e9, "unit": "GB/s",
+        "n_gpus": world, "steps": K, "warmup": args.warmup, "ms_per_step": total_ms_g / K,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u32",
+        "data": "synthetic", "impl": "ours",
+        "config": {"workload": w.name, "model": "jamba-like 4 attn + 28 mamba layers", "pool_gib": w.pool_bytes / W.GiB,
+                   "split": w.split, "migration_batch_size": w.migration_batch_size, "step_batch": w.concurrency,
+                   "warm_steps": WARM_STEPS, "running_mean": float(np.mean([len(r["run"]) for r in timed])),
+                   "tokens_mean": float(np.mean([int(r["lens"].sum()) for r in timed])),
+                   "l2": "inputs larger than L2 (each step moves GBs across a 4 GiB arena; per-layer outputs are distinct buffers)",
+                   "multi_gpu": "replicas only: one independent context per GPU, no collective"},
+        "allocator": {"ops_per_s": sums[1] / (sum(per["step"]) * 1e-3) * (world if world > 1 else 1),
+                      "us_per_step": step_avg_ms * 1e3, "ops_per_step": n_ops_total / K,
+                      "note": "avmp_step + avmp_translate, CUDA events around the two calls, rank 0's timing"},
+        "gather_kv": {"gbs": (kv_bytes / (K * m.n_attn_layers)) / (kv_avg_ms * 1e-3) / 1e9, "avg_ms": kv_avg_ms,
+                      "frac_of_peak": (kv_bytes / (K * m.n_attn_layers)) / (kv_avg_ms * 1e-3) / 1e9 / peak},
+        "migration": {"relocated_bytes_in_window": int(reloc_timed), "rebalances_total": st_c["n_rebalance"],
+                      "n_oom_total": st_c["n_oom"]},
+        "roofline": {"kernel": "ssm_copy_kernel<gather>", "bound": "hbm", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_source": f"MEASURED_PEAKS.json hbm_gbs ({peak_kind})",
+                     "frac_of_nominal_8000": achieved / 8000.0, "avg_launch_ms": ssm_avg_ms,
+                     "bytes_per_launch": ssm_launch_bytes,
+                     "traffic": None if NCU_TRAFFIC_RATIO is None else ssm_launch_bytes * NCU_TRAFFIC_RATIO},
+        "e2e": {"value": sums[0] / (e2e_ms_g * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms_g / K,
+                "h2d_bytes_per_step": sums[5] / K / world, "d2h_bytes_per_step": sums[6] / K / world,
+                "note": "ops and running list from host memory, statuses and row offsets back to the host every step; gathered batch buffers stay in HBM for the model's kernels"},
+        "gpu_launches": int(sums[4]),
+        "clocks": clocks,
+        "replay_matches_closed_loop": all(st_b[k] == stats_a[k] for k in stats_a),
+    }
+    return out
+
+
+# ---------------------------------------------------------------------------------------
+# the oracle on the host cores: cpu_baseline leg and the --impl reference arm
+# ---------------------------------------------------------------------------------------
+def run_oracle(args, n_sample_steps: int, budget_s: float = 25.0) -> dict:
+    from oracle.avmp_oracle import Oracle
+    w = W.config(args.workload, seed=args.seed)
+    m = w.model
+    o = Oracle.from_workload(w, with_store=True)
+    drv = W.ClosedLoopDriver(w)
+    while not drv.done and drv.step < WARM_STEPS:
+        ops = drv.next_batch()
+        drv.feed(o.step(ops))
+    # give every live unit real bytes (the stores are committed lazily)
+    run = drv.running_slots.astype(np.uint32)
+    rng = np.random.default_rng(0)
+    lens = drv.len[run]
+    for l in range(m.n_attn_layers):
+        kb = rng.integers(0, 256, (int(lens.sum()), m.kv_row_bytes), dtype=np.uint8)
+        o.scatter_kv(l, run, np.zeros(len(run), np.uint32), kb, kb)
+    sb = rng.integers(0, 256, (len(run), m.state_bytes), dtype=np.uint8)
+    cb = rng.integers(0, 256, (len(run), m.conv_bytes), dtype=np.uint8)
+    for l in range(m.n_ssm_layers):
+        o.scatter_ssm(l, run, sb, cb)
+    moved = n_ops = 0
+    t_alloc = t_total = 0.0
+    steps = 0
+    while steps < n_sample_steps and t_total < budget_s and not drv.done:
+        ops = drv.next_batch()
+        t0 = time.perf_counter()
+        st = o.step(ops)
+        t1 = time.perf_counter()
+        drv.feed(st)
+        run = drv.running_slots.astype(np.uint32)
+        lens = drv.len[run]
+        tot = int(lens.sum())
+        t2 = time.perf_counter()
+        tb = o.tables()
+        chain = tb["req_chain"].reshape(w.max_requests, w.max_pages)
+        handles = np.concatenate([chain[r, :tb["req_npages"][r]] for r in run] +
+                                 [tb["req_ssm"].reshape(w.max_requests, m.n_ssm_layers)[run].reshape(-1)])
+        t3 = time.perf_counter()
+        o.translate(handles)
+        for l in range(m.n_attn_layers):
+            o.gather_kv(l, run, tot)
+        for l in range(m.n_ssm_layers):
+            o.gather_ssm(l, run)
+        t4 = time.perf_counter()
+        b = step_bytes(m, len(run), tot, 0)
+        moved += b["kv"] + b["ssm"]
+        n_ops += len(ops)
+        t_alloc += t1 - t0
+        t_total += (t1 - t0) + (t4 - t3)
+        steps += 1
+    return {"value": moved / t_total / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+            "sample": f"{steps} consecutive engine steps of the same workload after {WARM_STEPS} warm steps "
+                      f"(allocator step + translate + all-layer gathers), {t_total:.1f} s of CPU work",
+            "allocator_ops_per_s": n_ops / t_alloc if t_alloc > 0 else None,
+            "ms_per_step": t_total / max(steps, 1) * 1e3, "steps": steps}
+
+
+def run_reference(args) -> dict:
+    w = W.config(args.workload, seed=args.seed)
+    n = max(1, min(args.steps, 8))
+    base = run_oracle(args, n_sample_steps=n, budget_s=120.0)
+    return {"metric": METRIC, "value": base["value"], "unit": "GB/s", "n_gpus": args.gpus, "steps": base["steps"],
+            "warmup": args.warmup, "ms_per_step": base["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "u32", "data": "synthetic", "impl": "reference",
+            "config": {"workload": w.name, "note": "the CPU oracle as it stands, single thread, bounded sample"},
+            "cpu_baseline": {k: base[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "allocator": {"ops_per_s": base["allocator_ops_per_s"]},
+            "e2e": {"value": base["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="short_uniform")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            print(json.dumps(run_reference(args)), flush=True)
+        return
+
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    out = run_ours(args, rank, world, local_rank)
+    if rank == 0:
+        if not args.no_cpu_baseline:
+            out["cpu_baseline"] = run_oracle(args, n_sample_steps=12)
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

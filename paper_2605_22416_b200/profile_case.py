@@ -1,0 +1,105 @@
+"""Small, self-contained launches of each kernel for profiling (a few GB on the device,
+a handful of launches): `python -m paper_2605_22416_b200.profile_case <case>`.
+
+Cases: ssm_gather, kv_gather, relocate, step.  Every case builds a context through the
+C ABI, brings it to a busy state with a few allocator steps and then launches the kernel
+of interest `--repeat` times on different layers, so every launch reads cold data.
+"""
+from __future__ import annotations
+
+import argparse
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import workloads as W
+
+
+def _dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a).view(np.uint8).reshape(-1)).cuda()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("case", choices=["ssm_gather", "kv_gather", "relocate", "step"])
+    ap.add_argument("--repeat", type=int, default=6)
+    ap.add_argument("--pool-gib", type=float, default=3.0)
+    args = ap.parse_args()
+    m = W.JAMBA_LIKE
+    pool = int(args.pool_gib * W.GiB)
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    if args.case in ("ssm_gather", "kv_gather", "step"):
+        split = 0.85 if args.case != "kv_gather" else 0.3
+        n_req = 150 if args.case != "kv_gather" else 48
+        tokens = 64 if args.case != "kv_gather" else 2048
+        ctx = B.Context(m, pool, split, 128, max_requests=256, max_pages=256)
+        ops = W.make_ops(W.OP_ADMIT, np.arange(n_req), tokens)
+        st = np.zeros(n_req, np.uint32)
+        ctx.step_host(ops, n_req, st)
+        assert (st == 0).all(), st
+        reqs = _dev(np.arange(n_req, dtype=np.uint32))
+        if args.case == "ssm_gather":
+            outs = [(torch.empty((n_req, m.state_bytes), dtype=torch.uint8, device="cuda"),
+                     torch.empty((n_req, m.conv_bytes), dtype=torch.uint8, device="cuda")) for _ in range(args.repeat)]
+            nbytes = 2 * n_req * (m.state_bytes + m.conv_bytes)
+            for i in range(args.repeat):
+                a, b = ev(), ev()
+                a.record()
+                ctx.gather_ssm(i % m.n_ssm_layers, reqs, n_req, outs[i][0], outs[i][1])
+                b.record()
+                torch.cuda.synchronize()
+                print(f"ssm_gather launch {i}: {a.elapsed_time(b) * 1e3:.1f} us, {nbytes / a.elapsed_time(b) / 1e6:.0f} GB/s")
+        elif args.case == "kv_gather":
+            tot = n_req * tokens
+            cu = torch.zeros(n_req + 1, dtype=torch.int32, device="cuda")
+            outs = [(torch.empty((tot, m.kv_row_bytes), dtype=torch.uint8, device="cuda"),
+                     torch.empty((tot, m.kv_row_bytes), dtype=torch.uint8, device="cuda")) for _ in range(min(args.repeat, 4))]
+            nbytes = 2 * tot * 2 * m.kv_row_bytes
+            for i in range(len(outs)):
+                a, b = ev(), ev()
+                a.record()
+                ctx.gather_kv(i % m.n_attn_layers, reqs, n_req, outs[i][0], outs[i][1], tot, cu)
+                b.record()
+                torch.cuda.synchronize()
+                print(f"kv_gather launch {i}: {a.elapsed_time(b) * 1e3:.1f} us, {nbytes / a.elapsed_time(b) / 1e6:.0f} GB/s")
+        else:
+            d_st = torch.zeros(n_req, dtype=torch.int32, device="cuda")
+            ext = _dev(W.make_ops(W.OP_EXTEND, np.arange(n_req), 1))
+            for i in range(args.repeat):
+                a, b = ev(), ev()
+                a.record()
+                ctx.step(ext, n_req, d_st)
+                b.record()
+                torch.cuda.synchronize()
+                print(f"step launch {i}: {a.elapsed_time(b) * 1e3:.1f} us for {n_req} ops")
+        print(ctx.stats())
+        ctx.close()
+        return
+
+    # relocate: fill the KV store, free every other long request so live pages are spread over
+    # the whole store, then exhaust the SSM store: the migration cedes the top of the KV store
+    # and must move the live pages it finds there.
+    B_units = 4096
+    ctx = B.Context(m, pool, 0.3, B_units, max_requests=512, max_pages=64, min_rebalance_interval_ops=1)
+    s0 = ctx.stats()
+    n_req = min(400, s0["cap_ssm"] // m.n_ssm_layers)
+    per = s0["cap_kv"] // n_req
+    st = np.zeros(n_req + 1, np.uint32)
+    ctx.step_host(W.make_ops(W.OP_ADMIT, np.arange(n_req), per * 16), n_req, st)
+    assert (st[:n_req] == 0).all()
+    ctx.step_host(W.make_ops(W.OP_FINISH, np.arange(0, n_req, 2), 0), n_req // 2, st)
+    a, b = ev(), ev()
+    a.record()
+    ctx.step_host(W.make_ops(W.OP_ADMIT, np.arange(0, n_req, 2)[:n_req // 2], 16), n_req // 2, st)
+    b.record()
+    torch.cuda.synchronize()
+    s = ctx.stats()
+    print(f"step with migration: {a.elapsed_time(b) * 1e3:.1f} us; relocated {s['relocated_blocks']} blocks, "
+          f"{s['relocated_bytes'] / 1e6:.1f} MB; rebalances {s['n_rebalance']}")
+    ctx.close()
+
+
+if __name__ == "__main__":
+    main()
