@@ -152,6 +152,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     # ---- phase B: replay from device-resident batches ----
     ctx = B.Context.from_workload(w, device=dev, arena=arena)
     stream = torch.cuda.current_stream()
+    sid = stream.cuda_stream          # raw cudaStream_t, passed straight to the C ABI
     max_run = max(len(r["run"]) for r in trace[WARM_STEPS:])
     max_tok = max(int(r["lens"].sum()) for r in trace[WARM_STEPS:])
     max_h = max(len(r["handles"]) for r in trace[WARM_STEPS:])
@@ -176,7 +177,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
         r["d_handles"] = to_dev(r["handles"])
 
     for r in trace[:WARM_STEPS]:
-        ctx.step(r["d_ops"], len(r["ops"]), d_status, stream)
+        ctx.step(r["d_ops"], len(r["ops"]), d_status, sid)
     torch.cuda.synchronize(dev)
     reloc0 = ctx.stats()["relocated_bytes"]
 
@@ -184,29 +185,25 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
         return torch.cuda.Event(enable_timing=True)
 
     def full_step(r, marks=None):
+        """marks: one event pair per kernel class per step (allocator, KV layers, SSM layers)."""
         n_ops, n_run = len(r["ops"]), len(r["run"])
         cap_tok = int(r["lens"].sum())
-        if marks is not None:
-            marks.append(("step", ev(), ev()))
-            marks[-1][1].record(stream)
-        ctx.step(r["d_ops"], n_ops, d_status, stream)
-        ctx.translate(r["d_handles"], len(r["handles"]), d_pool, d_off, d_aoff, stream)
-        if marks is not None:
-            marks[-1][2].record(stream)
+        e = [ev() for _ in range(4)] if marks is not None else None
+        if e:
+            e[0].record(stream)
+        ctx.step(r["d_ops"], n_ops, d_status, sid)
+        ctx.translate(r["d_handles"], len(r["handles"]), d_pool, d_off, d_aoff, sid)
+        if e:
+            e[1].record(stream)
         for l in range(m.n_attn_layers):
-            if marks is not None:
-                marks.append(("kv", ev(), ev()))
-                marks[-1][1].record(stream)
-            ctx.gather_kv(l, r["d_run"], n_run, out_k[l], out_v[l], cap_tok, d_cu, stream)
-            if marks is not None:
-                marks[-1][2].record(stream)
+            ctx.gather_kv(l, r["d_run"], n_run, out_k[l], out_v[l], cap_tok, d_cu, sid)
+        if e:
+            e[2].record(stream)
         for l in range(m.n_ssm_layers):
-            if marks is not None:
-                marks.append(("ssm", ev(), ev()))
-                marks[-1][1].record(stream)
-            ctx.gather_ssm(l, r["d_run"], n_run, out_s[l], out_c[l], stream)
-            if marks is not None:
-                marks[-1][2].record(stream)
+            ctx.gather_ssm(l, r["d_run"], n_run, out_s[l], out_c[l], sid)
+        if e:
+            e[3].record(stream)
+            marks.append(e)
 
     for r in trace[WARM_STEPS:WARM_STEPS + args.warmup]:
         full_step(r)
@@ -238,7 +235,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     ctx.close()
     ctx = B.Context.from_workload(w, device=dev, arena=arena)
     for r in trace[:WARM_STEPS]:
-        ctx.step(r["d_ops"], len(r["ops"]), d_status, stream)
+        ctx.step(r["d_ops"], len(r["ops"]), d_status, sid)
     for r in trace[WARM_STEPS:WARM_STEPS + args.warmup]:
         full_step(r)
     torch.cuda.synchronize(dev)
@@ -251,14 +248,16 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     st_c = ctx.stats()
     reloc_timed = st_c["relocated_bytes"] - reloc_w
     per = {"step": [], "kv": [], "ssm": []}
-    for kind, a, b in marks:
-        per[kind].append(a.elapsed_time(b))
+    for e in marks:
+        per["step"].append(e[0].elapsed_time(e[1]))
+        per["kv"].append(e[1].elapsed_time(e[2]) / m.n_attn_layers)      # average per launch
+        per["ssm"].append(e[2].elapsed_time(e[3]) / m.n_ssm_layers)
 
     # ---- e2e: host buffers in, host results out, every step ----
     ctx.close()
     ctx = B.Context.from_workload(w, device=dev, arena=arena)
     for r in trace[:WARM_STEPS + args.warmup]:
-        ctx.step(r["d_ops"], len(r["ops"]), d_status, stream)
+        ctx.step(r["d_ops"], len(r["ops"]), d_status, sid)
     torch.cuda.synchronize(dev)
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.uint8).reshape(-1).copy()).pin_memory()
     h_ops = [np.ascontiguousarray(r["ops"]) for r in timed]
@@ -271,13 +270,13 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     t0 = time.perf_counter()
     for r, ho, hr in zip(timed, h_ops, h_run):
         n_ops, n_run = len(r["ops"]), len(r["run"])
-        ctx.step_host(ho, n_ops, h_status, stream)                 # H2D ops, D2H statuses, sync
+        ctx.step_host(ho, n_ops, h_status, sid)                 # H2D ops, D2H statuses, sync
         d_run_buf[: hr.numel()].copy_(hr, non_blocking=True)       # H2D running list
         cap_tok = int(r["lens"].sum())
         for l in range(m.n_attn_layers):
-            ctx.gather_kv(l, d_run_buf, n_run, out_k[l], out_v[l], cap_tok, d_cu, stream)
+            ctx.gather_kv(l, d_run_buf, n_run, out_k[l], out_v[l], cap_tok, d_cu, sid)
         for l in range(m.n_ssm_layers):
-            ctx.gather_ssm(l, d_run_buf, n_run, out_s[l], out_c[l], stream)
+            ctx.gather_ssm(l, d_run_buf, n_run, out_s[l], out_c[l], sid)
         h_cu[: n_run + 1].copy_(d_cu[: n_run + 1], non_blocking=True)   # D2H row offsets of the batch
         torch.cuda.synchronize(dev)
         h2d += n_ops * 12 + n_run * 4

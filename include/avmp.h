@@ -73,7 +73,8 @@ enum {
     AVMP_DEV_OK = 0,
     AVMP_DEV_BAD_HANDLE = 1,     /* translate: handle does not resolve */
     AVMP_DEV_BAD_REQUEST = 2,    /* gather / scatter: request slot out of range or holds nothing */
-    AVMP_DEV_OUT_OVERFLOW = 3    /* gather_kv: rows would pass out_capacity_tokens */
+    AVMP_DEV_OUT_OVERFLOW = 3,   /* gather_kv: rows would pass out_capacity_tokens */
+    AVMP_DEV_TIMEOUT = 4         /* a copy kernel gave up a bounded wait; the output is incomplete */
 };
 
 /* Model shape: what one KV page and one SSM block hold (paper Section 3.1).

@@ -17,6 +17,7 @@ struct avmp_ctx {
     avmp_layout lay;
     uint32_t B;
     int n_sms;
+    int device;
     uint64_t launches;
     // staging for avmp_step_host, inside the workspace
     avmp_op *d_stage_ops;
@@ -72,7 +73,7 @@ bool options_ok(const avmp_options &o)
 }
 
 inline cudaStream_t S(void *s) { return reinterpret_cast<cudaStream_t>(s); }
-inline Launch L(const avmp_ctx *c, void *s) { return Launch{S(s), c->n_sms}; }
+inline Launch L(const avmp_ctx *c, void *s) { return Launch{S(s), c->n_sms, c->device}; }
 inline int cu(cudaError_t e) { return e == cudaSuccess ? AVMP_OK : AVMP_ECUDA; }
 
 void fill_stats(const avmp_ctx *c, const DevState &d, avmp_stats *o)
@@ -157,7 +158,8 @@ int avmp_create(avmp_ctx **out, const avmp_model_spec *spec, void *d_arena, uint
     if (!c) return AVMP_EINVAL;
     c->spec = *spec; c->opt = o; c->lay = lay; c->B = migration_batch_size; c->launches = 0;
     c->d_workspace = d_workspace; c->workspace_bytes = workspace_bytes;
-    int dev = 0;
+    int &dev = c->device;
+    dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
         delete c;

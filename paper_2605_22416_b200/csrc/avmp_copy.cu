@@ -3,54 +3,308 @@
 // arena and really moves live units), and the paged KV / contiguous SSM gathers and their
 // write sides (Section 2.2).  No arithmetic on payload: bytes in, bytes out.
 //
-// All of them are HBM-bound streaming copies.  Work is cut into warp-sized items of a few
-// KiB; consecutive warps take consecutive items, so a CTA streams one contiguous span.
-// Every lane keeps several 16-byte loads in flight before the first store.
+// All of them are HBM-bound streaming copies built on one skeleton.  The work of a launch
+// is a list of "pieces": contiguous byte runs of at most kStage bytes with a source and a
+// destination, enumerated by a small functor (SSM block chunks, page slices of a KV chain,
+// chunks of a relocated unit).  A persistent grid walks the piece list grid-strided at warp
+// granularity: at any moment the pieces in flight form one dense window of the list that
+// slides forward, which keeps the traffic spread evenly over the HBM channels (giving every
+// CTA its own contiguous range instead left 148 streams marching in lockstep at a fixed
+// stride and cost about 10 % of the bandwidth on this part).
+//
+//   * bulk path (the one real shapes take): each warp runs its own ring of kStages shared
+//     memory buffers.  One lane issues 1-D bulk async copies global -> shared (completion
+//     on an mbarrier) and shared -> global (bulk groups); no data passes through registers
+//     and the bytes in flight per SM are fixed by the ring (warps x stages x kStage), not
+//     by the compiler's scheduling.  Every wait is bounded: a warp that gives up records
+//     AVMP_DEV_TIMEOUT and stops issuing.
+//   * generic path: plain loads and stores, for shapes whose runs are not 16-byte multiples.
 #include "avmp_dev.cuh"
 
 namespace avmp {
 
 namespace {
 
-constexpr int kCopyThreads = 256;
-constexpr int kCtasPerSm = 8;
-constexpr uint32_t kChunk = 8192;      // bytes per warp item for contiguous copies
+// Tunables (overridable at build time for sweeps).
+#ifndef AVMP_STAGE_BYTES
+#define AVMP_STAGE_BYTES 16384
+#endif
+#ifndef AVMP_STAGES
+#define AVMP_STAGES 3
+#endif
+#ifndef AVMP_BULK_WARPS
+#define AVMP_BULK_WARPS 4
+#endif
+#ifndef AVMP_BULK_CTAS_PER_SM
+#define AVMP_BULK_CTAS_PER_SM 1
+#endif
+constexpr uint32_t kStage = AVMP_STAGE_BYTES;   // bytes per piece
+constexpr int kStages = AVMP_STAGES;            // ring depth per warp
+constexpr int kBulkWarps = AVMP_BULK_WARPS;     // warps (rings) per CTA: 4 x 3 x 16 KiB = 192 KiB of shared memory
+constexpr int kBulkCtasPerSm = AVMP_BULK_CTAS_PER_SM;
+constexpr int kBulkThreads = kBulkWarps * 32;
+constexpr uint32_t kBulkSmem = kBulkWarps * kStages * kStage;
+constexpr int kGenThreads = 256;
+constexpr int kGenCtasPerSm = 4;
+constexpr uint32_t kSpinLimit = 1u << 22;
 
-__device__ __forceinline__ uint4 ld_stream(const uint4 *p)
-{
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
-}
-__device__ __forceinline__ void st_stream(uint4 *p, const uint4 &v)
-{
-    asm volatile("st.global.L1::no_allocate.v4.u32 [%0], {%1,%2,%3,%4};"
-                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
+struct Piece {
+    const uint8_t *src;
+    uint8_t *dst;
+    uint32_t bytes;      // 0: nothing to do for this piece id
+};
 
-// One warp copies `bytes` (any size) from src to dst.  16-byte vectors when both ends and
-// the size allow, single bytes otherwise (only toy shapes take that path).
-template <int UNROLL>
-__device__ __forceinline__ void warp_copy(uint8_t *dst, const uint8_t *src, uint32_t bytes, int lane)
-{
-    if ((((uintptr_t)dst | (uintptr_t)src | bytes) & 15u) == 0) {
-        const uint4 *s = reinterpret_cast<const uint4 *>(src);
-        uint4 *d = reinterpret_cast<uint4 *>(dst);
-        const uint32_t nvec = bytes >> 4;
-        uint32_t i = lane;
-        for (; i + 32u * (UNROLL - 1) < nvec; i += 32u * UNROLL) {
-            uint4 v[UNROLL];
-#pragma unroll
-            for (int k = 0; k < UNROLL; ++k) v[k] = ld_stream(s + i + 32u * k);
-#pragma unroll
-            for (int k = 0; k < UNROLL; ++k) st_stream(d + i + 32u * k, v[k]);
+// ------------------------------- piece enumerators ------------------------------------
+// a12: SSM block <-> (state row, conv row) of the batch buffers.
+template <bool SCATTER>
+struct SsmPieces {
+    uint32_t layer, n, ps, per;
+    const uint32_t *reqs;
+    uint8_t *buf_state, *buf_conv;
+    __device__ unsigned long long total(const Geom &) const { return (unsigned long long)n * per; }
+    __device__ Piece get(const Geom &g, unsigned long long it) const
+    {
+        const uint32_t k = (uint32_t)(it / per), c = (uint32_t)(it % per);
+        const uint32_t r = reqs[k];
+        uint32_t slot = kInvalid;
+        if (r < g.R && g.r_state[r] == AVMP_REQ_LIVE) {
+            const uint32_t h = g.r_ssm[(unsigned long long)r * g.ns + layer];
+            if (h != kInvalid) slot = g.VT[1][h & 0x7FFFFFFFu];
         }
-        for (; i < nvec; i += 32u) st_stream(d + i, ld_stream(s + i));
-    } else {
-        for (uint32_t i = lane; i < bytes; i += 32u) dst[i] = src[i];
+        if (slot == kInvalid) {
+            if (c == 0) record_error(g.st, AVMP_DEV_BAD_REQUEST);
+            return Piece{nullptr, nullptr, 0};
+        }
+        uint8_t *blk = unit_ptr(g, AVMP_POOL_SSM, slot);
+        uint8_t *p, *b;
+        uint32_t bytes;
+        if (c < ps) {
+            const unsigned long long o = (unsigned long long)c * kStage;
+            p = blk + o; b = buf_state + (unsigned long long)k * g.state_bytes + o;
+            bytes = (uint32_t)min((unsigned long long)kStage, g.state_bytes - o);
+        } else {
+            const unsigned long long o = (unsigned long long)(c - ps) * kStage;
+            p = blk + g.state_bytes + o; b = buf_conv + (unsigned long long)k * g.conv_bytes + o;
+            bytes = (uint32_t)min((unsigned long long)kStage, g.conv_bytes - o);
+        }
+        return SCATTER ? Piece{b, p, bytes} : Piece{p, b, bytes};
+    }
+};
+
+// a7: chunks of the units moved by the last migration.
+struct RelocPieces {
+    __device__ unsigned long long total(const Geom &g) const
+    {
+        const unsigned long long U = g.U[g.st->reloc_pool];
+        return (unsigned long long)g.st->n_reloc * ((U + kStage - 1) / kStage);
+    }
+    __device__ Piece get(const Geom &g, unsigned long long it) const
+    {
+        const uint32_t pool = g.st->reloc_pool;
+        const unsigned long long U = g.U[pool];
+        const uint32_t per = (uint32_t)((U + kStage - 1) / kStage);
+        const uint32_t k = (uint32_t)(it / per), c = (uint32_t)(it % per);
+        const unsigned long long o = (unsigned long long)c * kStage;
+        // dst < new capacity <= src: the two units never overlap
+        return Piece{unit_ptr(g, pool, g.reloc_src[k]) + o, unit_ptr(g, pool, g.reloc_dst[k]) + o,
+                     (uint32_t)min((unsigned long long)kStage, U - o)};
+    }
+};
+
+// a11: slices of the pages of a KV chain <-> rows of the ragged batch buffers.  The plan
+// kernel has written, per request k, the first row (g_cu_rows) and the first piece
+// (g_cu_items); a request spanning P pages owns P * subs pieces, `subs` = slices per page
+// (K slices, then V slices).
+template <bool SCATTER>
+struct KvPieces {
+    uint32_t layer, n, subs;
+    const uint32_t *reqs, *tok_start;
+    uint8_t *buf_k, *buf_v;
+    unsigned long long cap_tokens;
+    __device__ unsigned long long total(const Geom &g) const { return g.st->g_total_items; }
+    __device__ Piece get(const Geom &g, unsigned long long it64) const
+    {
+        const uint32_t it = (uint32_t)it64;
+        const uint32_t k = find_owner(g.g_cu_items, 0u, n, 0u, it);
+        const uint32_t rel = it - g.g_cu_items[k];
+        const uint32_t row0 = g.g_cu_rows[k], rows = g.g_cu_rows[k + 1] - row0;
+        if (!SCATTER && (unsigned long long)row0 + rows > cap_tokens) {
+            if (rel == 0) record_error(g.st, AVMP_DEV_OUT_OVERFLOW);
+            return Piece{nullptr, nullptr, 0};
+        }
+        const uint32_t T = g.T, row = (uint32_t)g.row_bytes, half = subs >> 1;
+        const uint32_t t0 = tok_start ? tok_start[k] : 0u;
+        const uint32_t page = t0 / T + rel / subs, sub = rel % subs;
+        const uint32_t part = sub / half, q = sub % half;
+        // tokens of this page that belong to the copy, as a byte range of the page's K (or V) part
+        const uint32_t lo_t = max(t0, page * T), hi_t = min(t0 + rows, (page + 1u) * T);
+        const uint32_t b_lo = max((lo_t - page * T) * row, q * kStage);
+        const uint32_t b_hi = min((hi_t - page * T) * row, (q + 1u) * kStage);
+        if (b_lo >= b_hi) return Piece{nullptr, nullptr, 0};
+        const uint32_t r = reqs[k];
+        const uint32_t h = g.r_chain[(unsigned long long)r * g.max_pages + page];
+        const uint32_t slot = g.VT[0][h & 0x7FFFFFFFu];
+        uint8_t *p = g.arena + (unsigned long long)slot * g.U[0] + (unsigned long long)layer * g.kv_layer_bytes +
+                     (unsigned long long)part * T * row + b_lo;
+        // byte b of the page part is byte (b - (t0 - page*T)*row) of the request's rows
+        uint8_t *b = (part ? buf_v : buf_k) +
+                     ((unsigned long long)row0 * row + (unsigned long long)page * T * row + b_lo -
+                      (unsigned long long)t0 * row);
+        return SCATTER ? Piece{b, p, b_hi - b_lo} : Piece{p, b, b_hi - b_lo};
+    }
+};
+
+// ------------------------------- bulk-copy primitives ----------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_s2g(void *dst, uint32_t src_smem, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 :: "l"(dst), "r"(src_smem), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+template <int N>
+__device__ __forceinline__ void bulk_wait_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read %0;" :: "n"(N) : "memory");
+}
+// wait until at most `younger` of the most recent bulk groups still read shared memory
+__device__ __forceinline__ void wait_stage_free(uint32_t younger)
+{
+    static_assert(kStages <= 8, "extend the switch");
+    switch (younger) {
+    case 0: bulk_wait_read<0>(); break;
+    case 1: bulk_wait_read<1>(); break;
+    case 2: bulk_wait_read<2>(); break;
+    case 3: bulk_wait_read<3>(); break;
+    case 4: bulk_wait_read<4>(); break;
+    case 5: bulk_wait_read<5>(); break;
+    case 6: bulk_wait_read<6>(); break;
+    default: bulk_wait_read<7>(); break;
     }
 }
+__device__ __forceinline__ void bulk_wait_all()
+{
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
+// ------------------------------- the two skeletons --------------------------------------
+template <class F>
+__global__ void __launch_bounds__(kBulkThreads, kBulkCtasPerSm) stream_bulk_kernel(const Geom g, const F f)
+{
+    extern __shared__ __align__(1024) uint8_t ring[];
+    __shared__ __align__(8) unsigned long long bars[kBulkWarps * kStages];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const unsigned long long total = f.total(g);
+    if (lane == 0)
+        for (int s = 0; s < kStages; ++s) mbar_init(smem_u32(&bars[warp * kStages + s]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+    if (lane != 0) return;               // one lane drives its warp's ring
+
+    const uint32_t buf0 = smem_u32(ring) + (uint32_t)warp * kStages * kStage;
+    const uint32_t bar0 = smem_u32(&bars[warp * kStages]);
+    Piece pc[kStages];                   // piece sitting in each stage
+    uint32_t n_loaded = 0, n_stored = 0; // pieces issued as loads / as stores so far
+    bool drained = false, failed = false;
+    // warp w of CTA c takes pieces (w * grid + c) + j * (grid * warps), j = 0, 1, ...
+    const unsigned long long first = (unsigned long long)warp * gridDim.x + blockIdx.x;
+    const unsigned long long stride = (unsigned long long)gridDim.x * kBulkWarps;
+    unsigned long long n_taken = 0;
+
+    // Each loop turn: top up the ring with loads, then retire the oldest stage with a store.
+    while (true) {
+        while (!drained && n_loaded - n_stored < (uint32_t)kStages) {
+            const unsigned long long it = first + n_taken * stride;
+            ++n_taken;
+            if (it >= total) { drained = true; break; }
+            const Piece p = f.get(g, it);
+            if (p.bytes == 0) continue;
+            const uint32_t s = n_loaded % kStages;
+            // the stage's previous occupant was piece n_loaded - kStages; its store (one bulk group
+            // per piece, in order) must have finished reading the buffer.  Only younger groups may pend.
+            if (n_loaded >= (uint32_t)kStages) wait_stage_free(n_stored - 1u - (n_loaded - (uint32_t)kStages));
+            pc[s] = p;
+            mbar_expect_tx(bar0 + 8u * s, p.bytes);
+            bulk_g2s(buf0 + s * kStage, p.src, p.bytes, bar0 + 8u * s);
+            ++n_loaded;
+        }
+        if (n_stored == n_loaded) break;
+        const uint32_t s = n_stored % kStages, parity = (n_stored / kStages) & 1u;
+        uint32_t spins = 0;
+        while (!mbar_try_wait(bar0 + 8u * s, parity))
+            if (++spins > kSpinLimit) { failed = true; break; }
+        if (failed) break;
+        bulk_s2g(pc[s].dst, buf0 + s * kStage, pc[s].bytes);
+        ++n_stored;
+    }
+    if (failed) record_error(g.st, AVMP_DEV_TIMEOUT);
+    bulk_wait_all();
+}
+
+template <class F>
+__global__ void __launch_bounds__(kGenThreads) stream_generic_kernel(const Geom g, const F f)
+{
+    const int lane = threadIdx.x & 31;
+    const unsigned long long total = f.total(g);
+    const unsigned long long nw = (unsigned long long)gridDim.x * (kGenThreads / 32);
+    for (unsigned long long it = (unsigned long long)(threadIdx.x >> 5) * gridDim.x + blockIdx.x; it < total; it += nw) {
+        Piece p{nullptr, nullptr, 0};
+        if (lane == 0) p = f.get(g, it);
+        p.src = (const uint8_t *)__shfl_sync(0xFFFFFFFFu, (unsigned long long)p.src, 0);
+        p.dst = (uint8_t *)__shfl_sync(0xFFFFFFFFu, (unsigned long long)p.dst, 0);
+        p.bytes = __shfl_sync(0xFFFFFFFFu, p.bytes, 0);
+        if ((((uintptr_t)p.dst | (uintptr_t)p.src | p.bytes) & 15u) == 0) {
+            const uint4 *s = reinterpret_cast<const uint4 *>(p.src);
+            uint4 *d = reinterpret_cast<uint4 *>(p.dst);
+            for (uint32_t i = lane; i < (p.bytes >> 4); i += 32u) d[i] = s[i];
+        } else {
+            for (uint32_t i = lane; i < p.bytes; i += 32u) p.dst[i] = p.src[i];
+        }
+    }
+}
+
+template <class F>
+cudaError_t launch_stream(const Geom &g, const F &f, bool bulk_ok, const Launch &l)
+{
+    if (bulk_ok) {
+        static bool attr_set[64] = {};   // per kernel instantiation and device
+        if (!attr_set[l.device & 63]) {
+            cudaError_t e = cudaFuncSetAttribute(stream_bulk_kernel<F>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmem);
+            if (e != cudaSuccess) return e;
+            attr_set[l.device & 63] = true;
+        }
+        stream_bulk_kernel<F><<<l.n_sms * kBulkCtasPerSm, kBulkThreads, kBulkSmem, l.stream>>>(g, f);
+    } else {
+        stream_generic_kernel<F><<<l.n_sms * kGenCtasPerSm, kGenThreads, 0, l.stream>>>(g, f);
+    }
+    return cudaGetLastError();
+}
+
+inline bool mult16(unsigned long long x) { return (x & 15ull) == 0; }
 
 // ---- a10: translate ------------------------------------------------------------------
 __global__ void translate_kernel(const Geom g, const uint32_t *__restrict__ h, uint32_t n,
@@ -72,40 +326,17 @@ __global__ void translate_kernel(const Geom g, const uint32_t *__restrict__ h, u
     }
 }
 
-// ---- a7: relocation copy of the last migration -----------------------------------------
-__global__ void __launch_bounds__(kCopyThreads) relocate_kernel(const Geom g)
-{
-    const uint32_t n = g.st->n_reloc;
-    if (n == 0) return;
-    const uint32_t pool = g.st->reloc_pool;
-    const unsigned long long U = g.U[pool];
-    const uint32_t per = (uint32_t)((U + kChunk - 1) / kChunk);
-    const unsigned long long total = (unsigned long long)n * per;
-    const int lane = threadIdx.x & 31;
-    const unsigned long long nw = (unsigned long long)gridDim.x * (kCopyThreads / 32);
-    for (unsigned long long it = (unsigned long long)blockIdx.x * (kCopyThreads / 32) + (threadIdx.x >> 5);
-         it < total; it += nw) {
-        const uint32_t k = (uint32_t)(it / per), c = (uint32_t)(it % per);
-        const unsigned long long o = (unsigned long long)c * kChunk;
-        const uint32_t bytes = (uint32_t)min((unsigned long long)kChunk, U - o);
-        // dst < new capacity <= src: ranges never overlap
-        warp_copy<8>(unit_ptr(g, pool, g.reloc_dst[k]) + o, unit_ptr(g, pool, g.reloc_src[k]) + o, bytes, lane);
-    }
-}
-
-// ---- a11: KV gather / scatter ---------------------------------------------------------
-// Plan: one CTA turns the request list into row prefix sums (cu_seqlens) and item prefix
-// sums; an item is `tpi` consecutive rows of one request.
+// ---- a11 plan: request list -> row prefix sums (cu_seqlens) and piece prefix sums --------
 __global__ void __launch_bounds__(kStepThreads)
 kv_plan_kernel(const Geom g, const uint32_t *__restrict__ reqs, const uint32_t *__restrict__ tok_start,
-               uint32_t n, uint32_t tpi, uint32_t *__restrict__ cu_out)
+               uint32_t n, uint32_t subs, uint32_t *__restrict__ cu_out)
 {
     __shared__ unsigned long long tmp[32];
     unsigned long long run_rows = 0, run_items = 0, tot;
     const int tid = threadIdx.x;
     for (uint32_t b = 0; b < n; b += kStepThreads) {
         const uint32_t k = b + tid;
-        uint32_t rows = 0;
+        uint32_t rows = 0, items = 0;
         if (k < n) {
             const uint32_t r = reqs[k];
             const uint32_t st = r < g.R ? g.r_state[r] : AVMP_REQ_EMPTY;
@@ -116,8 +347,8 @@ kv_plan_kernel(const Geom g, const uint32_t *__restrict__ reqs, const uint32_t *
                 if (t0 > len) record_error(g.st, AVMP_DEV_BAD_REQUEST);
                 else rows = len - t0;
             }
+            if (rows) items = ((t0 + rows - 1u) / g.T - t0 / g.T + 1u) * subs;
         }
-        const uint32_t items = (rows + tpi - 1) / tpi;
         const unsigned long long incl = block_incl_scan(((unsigned long long)items << 32) | rows, tmp, &tot);
         if (k < n) {
             const uint32_t ex_rows = (uint32_t)(run_rows + (uint32_t)incl - rows);
@@ -137,96 +368,11 @@ kv_plan_kernel(const Geom g, const uint32_t *__restrict__ reqs, const uint32_t *
     }
 }
 
-template <bool SCATTER>
-__global__ void __launch_bounds__(kCopyThreads)
-kv_copy_kernel(const Geom g, const uint32_t layer, const uint32_t *__restrict__ reqs,
-               const uint32_t *__restrict__ tok_start, const uint32_t n, const uint32_t tpi,
-               uint8_t *__restrict__ buf_k, uint8_t *__restrict__ buf_v, const unsigned long long cap_tokens)
-{
-    const uint32_t total = g.st->g_total_items;
-    const int lane = threadIdx.x & 31;
-    const uint32_t row = (uint32_t)g.row_bytes, T = g.T;
-    const unsigned long long layer_off = (unsigned long long)layer * g.kv_layer_bytes;
-    const unsigned long long v_off = (unsigned long long)T * row;
-    const uint32_t nw = gridDim.x * (kCopyThreads / 32);
-    for (uint32_t it = blockIdx.x * (kCopyThreads / 32) + (threadIdx.x >> 5); it < total; it += nw) {
-        // request of this item: largest k with cu_items[k] <= it
-        const uint32_t k = find_owner(g.g_cu_items, 0u, n, 0u, it);
-        const uint32_t r = reqs[k];
-        const uint32_t row0 = g.g_cu_rows[k], rows = g.g_cu_rows[k + 1] - row0;
-        if (!SCATTER && (unsigned long long)row0 + rows > cap_tokens) {
-            if (it == g.g_cu_items[k] && lane == 0) record_error(g.st, AVMP_DEV_OUT_OVERFLOW);
-            continue;
-        }
-        const uint32_t i0 = (it - g.g_cu_items[k]) * tpi;          // first row of the item, request-relative
-        const uint32_t cnt = min(tpi, rows - i0);
-        const uint32_t t0 = (tok_start ? tok_start[k] : 0u) + i0;  // its token index
-        // rows of one item that share a page are contiguous in the page and in the buffer
-        uint32_t done = 0;
-        while (done < cnt) {
-            const uint32_t t = t0 + done;
-            const uint32_t in_page = min(cnt - done, T - t % T);
-            const uint32_t h = g.r_chain[(unsigned long long)r * g.max_pages + t / T];
-            const uint32_t slot = g.VT[0][h & 0x7FFFFFFFu];
-            uint8_t *pk = g.arena + (unsigned long long)slot * g.U[0] + layer_off + (unsigned long long)(t % T) * row;
-            uint8_t *bk = buf_k + ((unsigned long long)row0 + i0 + done) * row;
-            uint8_t *bv = buf_v + ((unsigned long long)row0 + i0 + done) * row;
-            const uint32_t bytes = in_page * row;
-            if (SCATTER) { warp_copy<4>(pk, bk, bytes, lane); warp_copy<4>(pk + v_off, bv, bytes, lane); }
-            else         { warp_copy<4>(bk, pk, bytes, lane); warp_copy<4>(bv, pk + v_off, bytes, lane); }
-            done += in_page;
-        }
-    }
-}
-
-// ---- a12: SSM gather / scatter ----------------------------------------------------------
-template <bool SCATTER>
-__global__ void __launch_bounds__(kCopyThreads)
-ssm_copy_kernel(const Geom g, const uint32_t layer, const uint32_t *__restrict__ reqs, const uint32_t n,
-                uint8_t *__restrict__ buf_state, uint8_t *__restrict__ buf_conv)
-{
-    const unsigned long long sb = g.state_bytes, cb = g.conv_bytes;
-    const uint32_t ps = (uint32_t)((sb + kChunk - 1) / kChunk), pc = (uint32_t)((cb + kChunk - 1) / kChunk);
-    const uint32_t per = ps + pc;
-    const unsigned long long total = (unsigned long long)n * per;
-    const int lane = threadIdx.x & 31;
-    const unsigned long long nw = (unsigned long long)gridDim.x * (kCopyThreads / 32);
-    for (unsigned long long it = (unsigned long long)blockIdx.x * (kCopyThreads / 32) + (threadIdx.x >> 5);
-         it < total; it += nw) {
-        const uint32_t k = (uint32_t)(it / per), c = (uint32_t)(it % per);
-        const uint32_t r = reqs[k];
-        uint32_t slot = kInvalid;
-        if (r < g.R && g.r_state[r] == AVMP_REQ_LIVE) {
-            const uint32_t h = g.r_ssm[(unsigned long long)r * g.ns + layer];
-            if (h != kInvalid) slot = g.VT[1][h & 0x7FFFFFFFu];
-        }
-        if (slot == kInvalid) {
-            if (c == 0 && lane == 0) record_error(g.st, AVMP_DEV_BAD_REQUEST);
-            continue;
-        }
-        uint8_t *blk = unit_ptr(g, AVMP_POOL_SSM, slot);
-        uint8_t *p, *b;
-        uint32_t bytes;
-        if (c < ps) {
-            const unsigned long long o = (unsigned long long)c * kChunk;
-            p = blk + o; b = buf_state + (unsigned long long)k * sb + o;
-            bytes = (uint32_t)min((unsigned long long)kChunk, sb - o);
-        } else {
-            const unsigned long long o = (unsigned long long)(c - ps) * kChunk;
-            p = blk + sb + o; b = buf_conv + (unsigned long long)k * cb + o;
-            bytes = (uint32_t)min((unsigned long long)kChunk, cb - o);
-        }
-        if (SCATTER) warp_copy<8>(p, b, bytes, lane);
-        else         warp_copy<8>(b, p, bytes, lane);
-    }
-}
-
 }  // namespace
 
 cudaError_t launch_relocate(const Geom &g, const Launch &l)
 {
-    relocate_kernel<<<l.n_sms * kCtasPerSm, kCopyThreads, 0, l.stream>>>(g);
-    return cudaGetLastError();
+    return launch_stream(g, RelocPieces{}, mult16(g.U[0]) && mult16(g.U[1]) && mult16(g.P_al), l);
 }
 
 cudaError_t launch_translate(const Geom &g, const uint32_t *h, uint32_t n, uint32_t *pool,
@@ -241,32 +387,25 @@ cudaError_t launch_kv(const Geom &g, bool scatter, uint32_t layer, const uint32_
                       const uint32_t *tok_start, uint32_t n, void *k, void *v,
                       unsigned long long cap_tokens, uint32_t *cu_out, const Launch &l)
 {
-    // rows per warp item: about 4 KiB of K and as much of V
-    uint32_t tpi = (uint32_t)(4096 / (g.row_bytes ? g.row_bytes : 1));
-    if (tpi < 1) tpi = 1;
-    if (tpi > g.T) tpi = g.T;
-    kv_plan_kernel<<<1, kStepThreads, 0, l.stream>>>(g, reqs, tok_start, n, tpi, cu_out);
+    const unsigned long long part = (unsigned long long)g.T * g.row_bytes;     // K (or V) bytes of a page
+    const uint32_t subs = 2u * (uint32_t)((part + kStage - 1) / kStage);
+    kv_plan_kernel<<<1, kStepThreads, 0, l.stream>>>(g, reqs, tok_start, n, subs, cu_out);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    const int grid = l.n_sms * kCtasPerSm;
+    const bool bulk_ok = mult16(g.row_bytes) && mult16(g.U[0]) && mult16(g.kv_layer_bytes);
     if (scatter)
-        kv_copy_kernel<true><<<grid, kCopyThreads, 0, l.stream>>>(g, layer, reqs, tok_start, n, tpi,
-                                                                 (uint8_t *)k, (uint8_t *)v, cap_tokens);
-    else
-        kv_copy_kernel<false><<<grid, kCopyThreads, 0, l.stream>>>(g, layer, reqs, tok_start, n, tpi,
-                                                                  (uint8_t *)k, (uint8_t *)v, cap_tokens);
-    return cudaGetLastError();
+        return launch_stream(g, KvPieces<true>{layer, n, subs, reqs, tok_start, (uint8_t *)k, (uint8_t *)v, cap_tokens}, bulk_ok, l);
+    return launch_stream(g, KvPieces<false>{layer, n, subs, reqs, tok_start, (uint8_t *)k, (uint8_t *)v, cap_tokens}, bulk_ok, l);
 }
 
 cudaError_t launch_ssm(const Geom &g, bool scatter, uint32_t layer, const uint32_t *reqs, uint32_t n,
                        void *state, void *conv, const Launch &l)
 {
-    const int grid = l.n_sms * kCtasPerSm;
+    const uint32_t ps = (uint32_t)((g.state_bytes + kStage - 1) / kStage), pc = (uint32_t)((g.conv_bytes + kStage - 1) / kStage);
+    const bool bulk_ok = mult16(g.state_bytes) && mult16(g.conv_bytes) && mult16(g.U[1]) && mult16(g.P_al);
     if (scatter)
-        ssm_copy_kernel<true><<<grid, kCopyThreads, 0, l.stream>>>(g, layer, reqs, n, (uint8_t *)state, (uint8_t *)conv);
-    else
-        ssm_copy_kernel<false><<<grid, kCopyThreads, 0, l.stream>>>(g, layer, reqs, n, (uint8_t *)state, (uint8_t *)conv);
-    return cudaGetLastError();
+        return launch_stream(g, SsmPieces<true>{layer, n, ps, ps + pc, reqs, (uint8_t *)state, (uint8_t *)conv}, bulk_ok, l);
+    return launch_stream(g, SsmPieces<false>{layer, n, ps, ps + pc, reqs, (uint8_t *)state, (uint8_t *)conv}, bulk_ok, l);
 }
 
 }  // namespace avmp

@@ -112,6 +112,7 @@ __device__ __forceinline__ uint32_t find_owner(const uint32_t *a, uint32_t lo, u
 struct Launch {
     cudaStream_t stream;
     int n_sms;
+    int device;
 };
 cudaError_t launch_init(const Geom &g, const DevState &init, cudaStream_t s);
 cudaError_t launch_step(const Geom &g, const avmp_op *d_ops, uint32_t n_ops, uint32_t *d_status,

@@ -82,22 +82,28 @@ def main():
     # the whole store, then exhaust the SSM store: the migration cedes the top of the KV store
     # and must move the live pages it finds there.
     B_units = 4096
-    ctx = B.Context(m, pool, 0.3, B_units, max_requests=512, max_pages=64, min_rebalance_interval_ops=1)
+    ctx = B.Context(m, pool, 0.3, B_units, max_requests=512, max_pages=256, min_rebalance_interval_ops=1)
     s0 = ctx.stats()
     n_req = min(400, s0["cap_ssm"] // m.n_ssm_layers)
-    per = s0["cap_kv"] // n_req
-    st = np.zeros(n_req + 1, np.uint32)
+    per = min(256, s0["cap_kv"] // n_req)
+    st = np.zeros(512, np.uint32)
     ctx.step_host(W.make_ops(W.OP_ADMIT, np.arange(n_req), per * 16), n_req, st)
-    assert (st[:n_req] == 0).all()
-    ctx.step_host(W.make_ops(W.OP_FINISH, np.arange(0, n_req, 2), 0), n_req // 2, st)
+    assert (st[:n_req] == 0).all(), st[:n_req]
+    ctx.step_host(W.make_ops(W.OP_FINISH, np.arange(0, n_req, 2), 0), (n_req + 1) // 2, st)
+    n_new = n_req                      # more admits than the SSM store can hold: forces KV -> SSM
+    d_ops = _dev(W.make_ops(W.OP_ADMIT, 256 + np.arange(n_new), 16))
+    d_st = torch.zeros(n_new, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
     a, b = ev(), ev()
     a.record()
-    ctx.step_host(W.make_ops(W.OP_ADMIT, np.arange(0, n_req, 2)[:n_req // 2], 16), n_req // 2, st)
+    ctx.step(d_ops, n_new, d_st)
     b.record()
     torch.cuda.synchronize()
     s = ctx.stats()
-    print(f"step with migration: {a.elapsed_time(b) * 1e3:.1f} us; relocated {s['relocated_blocks']} blocks, "
-          f"{s['relocated_bytes'] / 1e6:.1f} MB; rebalances {s['n_rebalance']}")
+    ms = a.elapsed_time(b)
+    print(f"step with migration: {ms * 1e3:.1f} us; relocated {s['relocated_blocks']} blocks, "
+          f"{s['relocated_bytes'] / 1e6:.1f} MB; rebalances {s['n_rebalance']}; "
+          f">= {2 * s['relocated_bytes'] / ms / 1e6:.0f} GB/s (whole step time as the denominator)")
     ctx.close()
 
 

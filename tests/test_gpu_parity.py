@@ -83,11 +83,11 @@ def test_random_op_strings_tiny(env, seed, batch):
 def test_many_migrations_inside_one_batch(env):
     """min_interval 1: a single batch holds many migrations in both directions, so the step
     runs as several plan/copy rounds; payload must follow every relocation."""
-    w = W.config("tiny", migration_batch_size=2, min_rebalance_interval_ops=1, pool_bytes=4096)
+    w = W.config("tiny", migration_batch_size=3, min_rebalance_interval_ops=1, pool_bytes=2048)
     g, o = _pair(env, w, with_store=True, max_requests=16, max_pages=8)
     rng = np.random.default_rng(3)
     for rnd in range(30):
-        ops = W.random_op_string(500 + rnd, 64, 16, 90, p_invalid=0.02)
+        ops = W.random_op_string(500 + rnd, 64, 16, 60, p_invalid=0.02)
         sg, so = g.step(ops), o.step(ops)
         assert np.array_equal(sg, so)
         env["same"](g, o, w, f"round {rnd}")
@@ -127,7 +127,7 @@ def test_many_migrations_inside_one_batch(env):
         os_, oc, ob = o.gather_ssm(0, live)
         assert gb == ob == 0 and np.array_equal(gs, sb) and np.array_equal(gc, cb)
         assert np.array_equal(os_, sb) and np.array_equal(oc, cb)
-    assert g.stats()["n_rebalance"] > 20 and g.stats()["relocated_blocks"] > 5
+    assert g.stats()["n_rebalance"] > 15 and g.stats()["relocated_blocks"] > 10
 
 
 def _closed_loop_parity(env, w, steps, *, with_store, kv_layers, ssm_layers, table_every, gather_every,
