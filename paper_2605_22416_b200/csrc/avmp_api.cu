@@ -10,21 +10,6 @@
 
 using namespace avmp;
 
-struct avmp_ctx {
-    Geom g;
-    avmp_model_spec spec;
-    avmp_options opt;
-    avmp_layout lay;
-    uint32_t B;
-    int n_sms;
-    int device;
-    uint64_t launches;
-    // staging for avmp_step_host, inside the workspace
-    avmp_op *d_stage_ops;
-    uint32_t *d_stage_status;
-    size_t workspace_bytes;
-    void *d_workspace;
-};
 
 namespace {
 

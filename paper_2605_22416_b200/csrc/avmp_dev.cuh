@@ -127,3 +127,22 @@ cudaError_t launch_ssm(const Geom &g, bool scatter, uint32_t layer, const uint32
                        void *state, void *conv, const Launch &l);
 
 }  // namespace avmp
+
+// The context behind the opaque avmp_ctx handle: a small host struct over the caller's arena
+// and workspace (global namespace: it is the C ABI's handle type).
+struct avmp_ctx {
+    avmp::Geom g;
+    avmp_model_spec spec;
+    avmp_options opt;
+    avmp_layout lay;
+    uint32_t B;
+    int n_sms;
+    int device;
+    uint64_t launches;
+    // staging for avmp_step_host, inside the workspace
+    avmp_op *d_stage_ops;
+    uint32_t *d_stage_status;
+    size_t workspace_bytes;
+    void *d_workspace;
+};
+
