@@ -48,7 +48,7 @@ extern "C" {
 #define AVMP_INVALID 0xFFFFFFFFu              /* no handle / no slot */
 #define AVMP_NONE64 0xFFFFFFFFFFFFFFFFull     /* no offset / "never" */
 
-enum { AVMP_OK = 0, AVMP_EINVAL = -1, AVMP_ENOSPC = -2, AVMP_ECUDA = -3 };
+enum { AVMP_OK = 0, AVMP_EINVAL = -1, AVMP_ENOSPC = -2, AVMP_ECUDA = -3, AVMP_ETOOBIG = -4 };
 enum { AVMP_POOL_KV = 0, AVMP_POOL_SSM = 1 };
 
 /* Operation kinds and flags (avmp_op). */
@@ -232,6 +232,23 @@ AVMP_API int avmp_scatter_kv(avmp_ctx *ctx, uint32_t attn_layer, const uint32_t 
                     const void *d_in_v, void *stream);
 AVMP_API int avmp_scatter_ssm(avmp_ctx *ctx, uint32_t ssm_layer, const uint32_t *d_reqs, uint32_t n_reqs,
                      const void *d_in_state, const void *d_in_conv, void *stream);
+
+/* (No counterpart in the paper: a deployment convenience.)  The same gather as avmp_gather_kv
+ * for callers that can neither allocate device memory nor lend the library scratch of their
+ * own -- e.g. code running after the process gave the whole card to a memory pool, or a
+ * plug-in that is only ever handed device pointers.  Inputs and outputs are still the
+ * caller's; the gather's planning arrays live in a fixed array inside the library
+ * (about 33 KB per GPU, held until the process exits), which limits the request list to
+ * AVMP_STATIC_GATHER_MAX_REQS entries: a longer list returns AVMP_ETOOBIG and does nothing.
+ * The context's device must be current.  The first call on a device resolves the array's
+ * device address (a host-side set-up step); make that first call before any stream capture.
+ * All calls on a device share the array: calls whose kernels may overlap on the GPU
+ * (different streams) race -- keep them on one stream or order them with events.  Results,
+ * error items and cu_seqlens are exactly those of avmp_gather_kv. */
+#define AVMP_STATIC_GATHER_MAX_REQS 4096
+AVMP_API int avmp_gather_kv_static(avmp_ctx *ctx, uint32_t attn_layer, const uint32_t *d_reqs, uint32_t n_reqs,
+                                   void *d_out_k, void *d_out_v, uint64_t out_capacity_tokens,
+                                   uint32_t *d_cu_seqlens, void *stream);
 
 /* Counters -> host.  Synchronises the stream. */
 AVMP_API int avmp_get_stats(avmp_ctx *ctx, avmp_stats *h_out, void *stream);

@@ -16,7 +16,8 @@ import torch
 
 from . import build as _build
 
-AVMP_OK, AVMP_EINVAL, AVMP_ENOSPC, AVMP_ECUDA = 0, -1, -2, -3
+AVMP_OK, AVMP_EINVAL, AVMP_ENOSPC, AVMP_ECUDA, AVMP_ETOOBIG = 0, -1, -2, -3, -4
+AVMP_STATIC_GATHER_MAX_REQS = 4096
 AVMP_INVALID = 0xFFFFFFFF
 AVMP_NONE64 = 0xFFFFFFFFFFFFFFFF
 
@@ -77,6 +78,7 @@ def _load():
         "avmp_step_host": (C.c_int, [vp, vp, C.c_uint32, vp, vp]),
         "avmp_translate": (C.c_int, [vp, vp, C.c_uint32, vp, vp, vp, vp]),
         "avmp_gather_kv": (C.c_int, [vp, C.c_uint32, vp, C.c_uint32, vp, vp, C.c_uint64, vp, vp]),
+        "avmp_gather_kv_static": (C.c_int, [vp, C.c_uint32, vp, C.c_uint32, vp, vp, C.c_uint64, vp, vp]),
         "avmp_gather_ssm": (C.c_int, [vp, C.c_uint32, vp, C.c_uint32, vp, vp, vp]),
         "avmp_scatter_kv": (C.c_int, [vp, C.c_uint32, vp, vp, C.c_uint32, vp, vp, vp]),
         "avmp_scatter_ssm": (C.c_int, [vp, C.c_uint32, vp, C.c_uint32, vp, vp, vp]),
@@ -174,6 +176,14 @@ def avmp_translate(ctx, d_handles, n, d_pool, d_offset, d_arena_offset=None, str
 def avmp_gather_kv(ctx, attn_layer, d_reqs, n_reqs, d_out_k, d_out_v, out_capacity_tokens, d_cu_seqlens, stream=None):
     _check(lib.avmp_gather_kv(ctx, attn_layer, _ptr(d_reqs), n_reqs, _ptr(d_out_k), _ptr(d_out_v),
                               out_capacity_tokens, _ptr(d_cu_seqlens), _stream(stream)), "avmp_gather_kv")
+
+
+def avmp_gather_kv_static(ctx, attn_layer, d_reqs, n_reqs, d_out_k, d_out_v, out_capacity_tokens, d_cu_seqlens,
+                          stream=None):
+    """avmp_gather_kv with the planning scratch inside the library (nothing lent, nothing allocated)."""
+    _check(lib.avmp_gather_kv_static(ctx, attn_layer, _ptr(d_reqs), n_reqs, _ptr(d_out_k), _ptr(d_out_v),
+                                     out_capacity_tokens, _ptr(d_cu_seqlens), _stream(stream)),
+           "avmp_gather_kv_static")
 
 
 def avmp_gather_ssm(ctx, ssm_layer, d_reqs, n_reqs, d_out_state, d_out_conv, stream=None):
@@ -318,6 +328,9 @@ class Context:
 
     def gather_kv(self, layer, d_reqs, n, d_out_k, d_out_v, cap_tokens, d_cu, stream=None):
         avmp_gather_kv(self.handle, layer, d_reqs, n, d_out_k, d_out_v, cap_tokens, d_cu, stream)
+
+    def gather_kv_static(self, layer, d_reqs, n, d_out_k, d_out_v, cap_tokens, d_cu, stream=None):
+        avmp_gather_kv_static(self.handle, layer, d_reqs, n, d_out_k, d_out_v, cap_tokens, d_cu, stream)
 
     def gather_ssm(self, layer, d_reqs, n, d_out_state, d_out_conv, stream=None):
         avmp_gather_ssm(self.handle, layer, d_reqs, n, d_out_state, d_out_conv, stream)

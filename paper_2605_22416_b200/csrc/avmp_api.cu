@@ -368,6 +368,7 @@ const char *avmp_error_string(int code)
     case AVMP_EINVAL: return "invalid argument";
     case AVMP_ENOSPC: return "workspace too small";
     case AVMP_ECUDA: return "CUDA runtime error";
+    case AVMP_ETOOBIG: return "request list longer than the fixed in-library scratch allows (AVMP_STATIC_GATHER_MAX_REQS)";
     default: return "unknown error";
     }
 }
