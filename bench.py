@@ -150,17 +150,18 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     ctx.close()
 
     # ---- phase B: replay from device-resident batches ----
-    ctx = B.Context.from_workload(w, device=dev, arena=arena)
     stream = torch.cuda.current_stream()
     sid = stream.cuda_stream          # raw cudaStream_t, passed straight to the C ABI
     max_run = max(len(r["run"]) for r in trace[WARM_STEPS:])
     max_tok = max(int(r["lens"].sum()) for r in trace[WARM_STEPS:])
     max_h = max(len(r["handles"]) for r in trace[WARM_STEPS:])
     d_status = torch.zeros(w.concurrency * 2 + 16, dtype=torch.int32, device=dev)
-    out_k = [torch.empty((max_tok, m.kv_row_bytes), dtype=torch.uint8, device=dev) for _ in range(m.n_attn_layers)]
-    out_v = [torch.empty((max_tok, m.kv_row_bytes), dtype=torch.uint8, device=dev) for _ in range(m.n_attn_layers)]
-    out_s = [torch.empty((max_run, m.state_bytes), dtype=torch.uint8, device=dev) for _ in range(m.n_ssm_layers)]
-    out_c = [torch.empty((max_run, m.conv_bytes), dtype=torch.uint8, device=dev) for _ in range(m.n_ssm_layers)]
+    # batch buffers: one slab per kind, [layer][row]; every layer has its own rows (no buffer reuse)
+    out_k = torch.empty((m.n_attn_layers, max_tok, m.kv_row_bytes), dtype=torch.uint8, device=dev)
+    out_v = torch.empty((m.n_attn_layers, max_tok, m.kv_row_bytes), dtype=torch.uint8, device=dev)
+    out_s = torch.empty((m.n_ssm_layers, max_run, m.state_bytes), dtype=torch.uint8, device=dev)
+    out_c = torch.empty((m.n_ssm_layers, max_run, m.conv_bytes), dtype=torch.uint8, device=dev)
+    kv_stride, s_stride, c_stride = max_tok * m.kv_row_bytes, max_run * m.state_bytes, max_run * m.conv_bytes
     d_cu = torch.zeros(max_run + 1, dtype=torch.int32, device=dev)
     d_pool = torch.zeros(max_h, dtype=torch.int32, device=dev)
     d_off = torch.zeros(max_h, dtype=torch.int64, device=dev)
@@ -176,40 +177,56 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
         r["d_run"] = to_dev(r["run"])
         r["d_handles"] = to_dev(r["handles"])
 
-    for r in trace[:WARM_STEPS]:
-        ctx.step(r["d_ops"], len(r["ops"]), d_status, sid)
-    torch.cuda.synchronize(dev)
-    reloc0 = ctx.stats()["relocated_bytes"]
-
     def ev():
         return torch.cuda.Event(enable_timing=True)
 
-    def full_step(r, marks=None):
-        """marks: one event pair per kernel class per step (allocator, KV layers, SSM layers)."""
+    def fresh_context(full_warmup=True):
+        """A new context over the same arena, replayed up to the start of the timed window."""
+        c = B.Context.from_workload(w, device=dev, arena=arena)
+        for r in trace[:WARM_STEPS]:
+            c.step(r["d_ops"], len(r["ops"]), d_status, sid)
+        for r in trace[WARM_STEPS:WARM_STEPS + args.warmup]:
+            if full_warmup:
+                full_step(c, r)
+            else:
+                c.step(r["d_ops"], len(r["ops"]), d_status, sid)
+        torch.cuda.synchronize(dev)
+        return c
+
+    def full_step(c, r, marks=None, per_layer=False, d_run=None):
+        """One engine step.  marks: one event pair per kernel class (allocator, KV, SSM).
+        per_layer: one launch per layer instead of one launch for all layers."""
         n_ops, n_run = len(r["ops"]), len(r["run"])
         cap_tok = int(r["lens"].sum())
+        run = r["d_run"] if d_run is None else d_run
         e = [ev() for _ in range(4)] if marks is not None else None
         if e:
             e[0].record(stream)
-        ctx.step(r["d_ops"], n_ops, d_status, sid)
-        ctx.translate(r["d_handles"], len(r["handles"]), d_pool, d_off, d_aoff, sid)
+        c.step(r["d_ops"], n_ops, d_status, sid)
+        c.translate(r["d_handles"], len(r["handles"]), d_pool, d_off, d_aoff, sid)
         if e:
             e[1].record(stream)
-        for l in range(m.n_attn_layers):
-            ctx.gather_kv(l, r["d_run"], n_run, out_k[l], out_v[l], cap_tok, d_cu, sid)
+        if per_layer:
+            for l in range(m.n_attn_layers):
+                c.gather_kv(l, run, n_run, out_k[l], out_v[l], cap_tok, d_cu, sid)
+        else:
+            c.gather_kv_layers(0, m.n_attn_layers, run, n_run, out_k, out_v, kv_stride, cap_tok, d_cu, sid)
         if e:
             e[2].record(stream)
-        for l in range(m.n_ssm_layers):
-            ctx.gather_ssm(l, r["d_run"], n_run, out_s[l], out_c[l], sid)
+        if per_layer:
+            for l in range(m.n_ssm_layers):
+                c.gather_ssm(l, run, n_run, out_s[l], out_c[l], sid)
+        else:
+            c.gather_ssm_layers(0, m.n_ssm_layers, run, n_run, out_s, s_stride, out_c, c_stride, sid)
         if e:
             e[3].record(stream)
             marks.append(e)
 
-    for r in trace[WARM_STEPS:WARM_STEPS + args.warmup]:
-        full_step(r)
     timed = trace[WARM_STEPS + args.warmup:]
 
-    # ---- timed region 1: K whole steps, one pair of events, no per-kernel events inside ----
+    # ---- timed region 1: K whole steps, one pair of events, nothing else on the stream ----
+    ctx = fresh_context()
+    reloc0 = ctx.stats()["relocated_bytes"]
     if world > 1:
         import torch.distributed as dist
         dist.barrier()
@@ -220,7 +237,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     e0, e1 = ev(), ev()
     e0.record(stream)
     for r in timed:
-        full_step(r)
+        full_step(ctx, r)
     e1.record(stream)
     torch.cuda.synchronize(dev)
     if world > 1:
@@ -228,37 +245,30 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     total_ms = e0.elapsed_time(e1)
     launches = ctx.launch_count() - launches0
     st_b = ctx.stats()
-    reloc_bytes = st_b["relocated_bytes"] - reloc0   # includes warm-up steps' relocations: subtract below
-
-    # ---- timed region 2 (same steps cannot be replayed: state moved on); per-kernel durations come
-    # from a second replay of the same window on a fresh context, with events around each call ----
+    reloc_timed = st_b["relocated_bytes"] - reloc0
     ctx.close()
-    ctx = B.Context.from_workload(w, device=dev, arena=arena)
-    for r in trace[:WARM_STEPS]:
-        ctx.step(r["d_ops"], len(r["ops"]), d_status, sid)
-    for r in trace[WARM_STEPS:WARM_STEPS + args.warmup]:
-        full_step(r)
-    torch.cuda.synchronize(dev)
-    reloc_w = ctx.stats()["relocated_bytes"]
-    marks = []
-    for r in timed:
-        full_step(r, marks)
-    torch.cuda.synchronize(dev)
+
+    # ---- region 2: the same window again with one event pair per kernel class and step ----
+    def timed_classes(per_layer):
+        c = fresh_context()
+        marks = []
+        for r in timed:
+            full_step(c, r, marks, per_layer=per_layer)
+        torch.cuda.synchronize(dev)
+        st = c.stats()
+        c.close()
+        nl_kv = m.n_attn_layers if per_layer else 1
+        nl_ssm = m.n_ssm_layers if per_layer else 1
+        return ({"step": [e[0].elapsed_time(e[1]) for e in marks],
+                 "kv": [e[1].elapsed_time(e[2]) / nl_kv for e in marks],       # average per launch
+                 "ssm": [e[2].elapsed_time(e[3]) / nl_ssm for e in marks]}, st)
+
+    per, st_c = timed_classes(per_layer=False)
+    per_l, _ = timed_classes(per_layer=True)
     clocks = sampler.stop()
-    st_c = ctx.stats()
-    reloc_timed = st_c["relocated_bytes"] - reloc_w
-    per = {"step": [], "kv": [], "ssm": []}
-    for e in marks:
-        per["step"].append(e[0].elapsed_time(e[1]))
-        per["kv"].append(e[1].elapsed_time(e[2]) / m.n_attn_layers)      # average per launch
-        per["ssm"].append(e[2].elapsed_time(e[3]) / m.n_ssm_layers)
 
     # ---- e2e: host buffers in, host results out, every step ----
-    ctx.close()
-    ctx = B.Context.from_workload(w, device=dev, arena=arena)
-    for r in trace[:WARM_STEPS + args.warmup]:
-        ctx.step(r["d_ops"], len(r["ops"]), d_status, sid)
-    torch.cuda.synchronize(dev)
+    ctx = fresh_context(full_warmup=False)
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.uint8).reshape(-1).copy()).pin_memory()
     h_ops = [np.ascontiguousarray(r["ops"]) for r in timed]
     h_run = [pin(r["run"]) for r in timed]
@@ -270,13 +280,11 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     t0 = time.perf_counter()
     for r, ho, hr in zip(timed, h_ops, h_run):
         n_ops, n_run = len(r["ops"]), len(r["run"])
-        ctx.step_host(ho, n_ops, h_status, sid)                 # H2D ops, D2H statuses, sync
+        ctx.step_host(ho, n_ops, h_status, sid)                    # H2D ops, D2H statuses, sync
         d_run_buf[: hr.numel()].copy_(hr, non_blocking=True)       # H2D running list
         cap_tok = int(r["lens"].sum())
-        for l in range(m.n_attn_layers):
-            ctx.gather_kv(l, d_run_buf, n_run, out_k[l], out_v[l], cap_tok, d_cu, sid)
-        for l in range(m.n_ssm_layers):
-            ctx.gather_ssm(l, d_run_buf, n_run, out_s[l], out_c[l], sid)
+        ctx.gather_kv_layers(0, m.n_attn_layers, d_run_buf, n_run, out_k, out_v, kv_stride, cap_tok, d_cu, sid)
+        ctx.gather_ssm_layers(0, m.n_ssm_layers, d_run_buf, n_run, out_s, s_stride, out_c, c_stride, sid)
         h_cu[: n_run + 1].copy_(d_cu[: n_run + 1], non_blocking=True)   # D2H row offsets of the batch
         torch.cuda.synchronize(dev)
         h2d += n_ops * 12 + n_run * 4
@@ -296,11 +304,14 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     e2e_ms_g, _ = reduce_over_ranks(e2e_ms, np.zeros(1), world)
     peak, peak_kind = _peaks()
 
-    ssm_launch_bytes = ssm_bytes / (K * m.n_ssm_layers)
+    ssm_launch_bytes = ssm_bytes / K                       # one launch gathers all SSM layers of a step
     ssm_avg_ms = float(np.mean(per["ssm"]))
     achieved = ssm_launch_bytes / (ssm_avg_ms * 1e-3) / 1e9
+    kv_launch_bytes = kv_bytes / K
     kv_avg_ms = float(np.mean(per["kv"]))
     step_avg_ms = float(np.mean(per["step"]))
+    pl_ssm = (ssm_bytes / (K * m.n_ssm_layers)) / (float(np.mean(per_l["ssm"])) * 1e-3) / 1e9
+    pl_kv = (kv_bytes / (K * m.n_attn_layers)) / (float(np.mean(per_l["kv"])) * 1e-3) / 1e9
     out = {
         "metric": METRIC, "value": sums[0] / (total_ms_g * 1e-3) / 1e9, "unit": "GB/s",
         "n_gpus": world, "steps": K, "warmup": args.warmup, "ms_per_step": total_ms_g / K,
@@ -315,18 +326,23 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
         "allocator": {"ops_per_s": sums[1] / (sum(per["step"]) * 1e-3) * (world if world > 1 else 1),
                       "us_per_step": step_avg_ms * 1e3, "ops_per_step": n_ops_total / K,
                       "note": "avmp_step + avmp_translate, CUDA events around the two calls, rank 0's timing"},
-        "gather_kv": {"gbs": (kv_bytes / (K * m.n_attn_layers)) / (kv_avg_ms * 1e-3) / 1e9, "avg_ms": kv_avg_ms,
-                      "frac_of_peak": (kv_bytes / (K * m.n_attn_layers)) / (kv_avg_ms * 1e-3) / 1e9 / peak},
+        "gather_kv": {"gbs": kv_launch_bytes / (kv_avg_ms * 1e-3) / 1e9, "avg_launch_ms": kv_avg_ms,
+                      "frac_of_peak": kv_launch_bytes / (kv_avg_ms * 1e-3) / 1e9 / peak,
+                      "note": "avmp_gather_kv_layers: plan kernel + one copy launch for all attention layers"},
+        "per_layer_launches": {"gather_ssm_gbs": pl_ssm, "gather_ssm_frac_of_peak": pl_ssm / peak,
+                               "gather_ssm_avg_launch_ms": float(np.mean(per_l["ssm"])),
+                               "gather_kv_gbs": pl_kv, "gather_kv_frac_of_peak": pl_kv / peak,
+                               "note": "same window with avmp_gather_ssm / avmp_gather_kv called once per layer"},
         "migration": {"relocated_bytes_in_window": int(reloc_timed), "rebalances_total": st_c["n_rebalance"],
                       "n_oom_total": st_c["n_oom"]},
-        "roofline": {"kernel": "ssm_copy_kernel<gather>", "bound": "hbm", "achieved": achieved, "peak": peak,
+        "roofline": {"kernel": "stream_bulk_kernel<SsmPieces<gather>> (avmp_gather_ssm_layers, all SSM layers in one launch)", "bound": "hbm", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": f"MEASURED_PEAKS.json hbm_gbs ({peak_kind})",
                      "frac_of_nominal_8000": achieved / 8000.0, "avg_launch_ms": ssm_avg_ms,
                      "bytes_per_launch": ssm_launch_bytes,
                      "traffic": None if NCU_TRAFFIC_RATIO is None else ssm_launch_bytes * NCU_TRAFFIC_RATIO},
         "e2e": {"value": sums[0] / (e2e_ms_g * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms_g / K,
                 "h2d_bytes_per_step": sums[5] / K / world, "d2h_bytes_per_step": sums[6] / K / world,
-                "note": "ops and running list from host memory, statuses and row offsets back to the host every step; gathered batch buffers stay in HBM for the model's kernels"},
+                "note": "ops and running list from pinned/pageable host memory, statuses and row offsets back to the host every step; gathered batch buffers stay in HBM for the model's kernels"},
         "gpu_launches": int(sums[4]),
         "clocks": clocks,
         "replay_matches_closed_loop": all(st_b[k] == stats_a[k] for k in stats_a),

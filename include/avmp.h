@@ -224,6 +224,19 @@ AVMP_API int avmp_gather_kv(avmp_ctx *ctx, uint32_t attn_layer, const uint32_t *
 AVMP_API int avmp_gather_ssm(avmp_ctx *ctx, uint32_t ssm_layer, const uint32_t *d_reqs, uint32_t n_reqs,
                     void *d_out_state, void *d_out_conv, void *stream);
 
+/* The two gathers for `n_layers` consecutive layers in ONE launch (same results as calling the
+ * single-layer entry once per layer; one launch instead of n_layers removes the per-launch ramp
+ * and tail, which is most of what separates a 250 MB gather from the HBM roofline).  Layer
+ * first_layer + l writes to the given buffers advanced by l * stride bytes; strides are multiples
+ * of 16 and at least one layer's worth (out_capacity_tokens rows for KV, n_reqs blocks for SSM).
+ * d_cu_seqlens is shared by all layers. */
+AVMP_API int avmp_gather_kv_layers(avmp_ctx *ctx, uint32_t first_layer, uint32_t n_layers, const uint32_t *d_reqs,
+                                   uint32_t n_reqs, void *d_out_k, void *d_out_v, uint64_t layer_stride_bytes,
+                                   uint64_t out_capacity_tokens, uint32_t *d_cu_seqlens, void *stream);
+AVMP_API int avmp_gather_ssm_layers(avmp_ctx *ctx, uint32_t first_layer, uint32_t n_layers, const uint32_t *d_reqs,
+                                    uint32_t n_reqs, void *d_out_state, uint64_t state_layer_stride_bytes,
+                                    void *d_out_conv, uint64_t conv_layer_stride_bytes, void *stream);
+
 /* Write side of the two gathers (what the model's kernels do after a step).  Tokens
  * [d_tok_start[k], len_k) of request k are read from rows cu[k].. of d_in_k / d_in_v, cu being
  * the prefix sum of (len_k - d_tok_start[k]); d_tok_start == NULL means 0. */

@@ -80,6 +80,8 @@ def _load():
         "avmp_gather_kv": (C.c_int, [vp, C.c_uint32, vp, C.c_uint32, vp, vp, C.c_uint64, vp, vp]),
         "avmp_gather_kv_static": (C.c_int, [vp, C.c_uint32, vp, C.c_uint32, vp, vp, C.c_uint64, vp, vp]),
         "avmp_gather_ssm": (C.c_int, [vp, C.c_uint32, vp, C.c_uint32, vp, vp, vp]),
+        "avmp_gather_kv_layers": (C.c_int, [vp, C.c_uint32, C.c_uint32, vp, C.c_uint32, vp, vp, C.c_uint64, C.c_uint64, vp, vp]),
+        "avmp_gather_ssm_layers": (C.c_int, [vp, C.c_uint32, C.c_uint32, vp, C.c_uint32, vp, C.c_uint64, vp, C.c_uint64, vp]),
         "avmp_scatter_kv": (C.c_int, [vp, C.c_uint32, vp, vp, C.c_uint32, vp, vp, vp]),
         "avmp_scatter_ssm": (C.c_int, [vp, C.c_uint32, vp, C.c_uint32, vp, vp, vp]),
         "avmp_get_stats": (C.c_int, [vp, C.POINTER(avmp_stats), vp]),
@@ -189,6 +191,20 @@ def avmp_gather_kv_static(ctx, attn_layer, d_reqs, n_reqs, d_out_k, d_out_v, out
 def avmp_gather_ssm(ctx, ssm_layer, d_reqs, n_reqs, d_out_state, d_out_conv, stream=None):
     _check(lib.avmp_gather_ssm(ctx, ssm_layer, _ptr(d_reqs), n_reqs, _ptr(d_out_state), _ptr(d_out_conv),
                                _stream(stream)), "avmp_gather_ssm")
+
+
+def avmp_gather_kv_layers(ctx, first_layer, n_layers, d_reqs, n_reqs, d_out_k, d_out_v, layer_stride_bytes,
+                          out_capacity_tokens, d_cu_seqlens, stream=None):
+    _check(lib.avmp_gather_kv_layers(ctx, first_layer, n_layers, _ptr(d_reqs), n_reqs, _ptr(d_out_k), _ptr(d_out_v),
+                                     layer_stride_bytes, out_capacity_tokens, _ptr(d_cu_seqlens), _stream(stream)),
+           "avmp_gather_kv_layers")
+
+
+def avmp_gather_ssm_layers(ctx, first_layer, n_layers, d_reqs, n_reqs, d_out_state, state_layer_stride_bytes,
+                           d_out_conv, conv_layer_stride_bytes, stream=None):
+    _check(lib.avmp_gather_ssm_layers(ctx, first_layer, n_layers, _ptr(d_reqs), n_reqs, _ptr(d_out_state),
+                                      state_layer_stride_bytes, _ptr(d_out_conv), conv_layer_stride_bytes,
+                                      _stream(stream)), "avmp_gather_ssm_layers")
 
 
 def avmp_scatter_kv(ctx, attn_layer, d_reqs, d_tok_start, n_reqs, d_in_k, d_in_v, stream=None):
@@ -334,6 +350,16 @@ class Context:
 
     def gather_ssm(self, layer, d_reqs, n, d_out_state, d_out_conv, stream=None):
         avmp_gather_ssm(self.handle, layer, d_reqs, n, d_out_state, d_out_conv, stream)
+
+    def gather_kv_layers(self, first_layer, n_layers, d_reqs, n, d_out_k, d_out_v, layer_stride, cap_tokens, d_cu,
+                         stream=None):
+        avmp_gather_kv_layers(self.handle, first_layer, n_layers, d_reqs, n, d_out_k, d_out_v, layer_stride,
+                              cap_tokens, d_cu, stream)
+
+    def gather_ssm_layers(self, first_layer, n_layers, d_reqs, n, d_out_state, state_stride, d_out_conv,
+                          conv_stride, stream=None):
+        avmp_gather_ssm_layers(self.handle, first_layer, n_layers, d_reqs, n, d_out_state, state_stride,
+                               d_out_conv, conv_stride, stream)
 
     def scatter_kv(self, layer, d_reqs, d_tok_start, n, d_in_k, d_in_v, stream=None):
         avmp_scatter_kv(self.handle, layer, d_reqs, d_tok_start, n, d_in_k, d_in_v, stream)

@@ -248,7 +248,7 @@ int avmp_gather_kv(avmp_ctx *c, uint32_t layer, const uint32_t *d_reqs, uint32_t
     if (n && (!d_reqs || !d_out_k || !d_out_v)) return AVMP_EINVAL;
     if (((uintptr_t)d_out_k | (uintptr_t)d_out_v) & 15) return AVMP_EINVAL;
     c->launches += 2;
-    return cu(launch_kv(c->g, false, layer, d_reqs, nullptr, n, d_out_k, d_out_v, cap_tokens, d_cu, L(c, stream)));
+    return cu(launch_kv(c->g, false, layer, 1, d_reqs, nullptr, n, d_out_k, d_out_v, 0, cap_tokens, d_cu, L(c, stream)));
 }
 
 int avmp_scatter_kv(avmp_ctx *c, uint32_t layer, const uint32_t *d_reqs, const uint32_t *d_tok_start,
@@ -258,8 +258,8 @@ int avmp_scatter_kv(avmp_ctx *c, uint32_t layer, const uint32_t *d_reqs, const u
     if (n == 0) return AVMP_OK;
     if (!d_reqs || !d_in_k || !d_in_v || (((uintptr_t)d_in_k | (uintptr_t)d_in_v) & 15)) return AVMP_EINVAL;
     c->launches += 2;
-    return cu(launch_kv(c->g, true, layer, d_reqs, d_tok_start, n, const_cast<void *>(d_in_k),
-                        const_cast<void *>(d_in_v), ~0ull, nullptr, L(c, stream)));
+    return cu(launch_kv(c->g, true, layer, 1, d_reqs, d_tok_start, n, const_cast<void *>(d_in_k),
+                        const_cast<void *>(d_in_v), 0, ~0ull, nullptr, L(c, stream)));
 }
 
 int avmp_gather_ssm(avmp_ctx *c, uint32_t layer, const uint32_t *d_reqs, uint32_t n, void *d_out_state,
@@ -269,7 +269,7 @@ int avmp_gather_ssm(avmp_ctx *c, uint32_t layer, const uint32_t *d_reqs, uint32_
     if (n == 0) return AVMP_OK;
     if (!d_reqs || !d_out_state || !d_out_conv || (((uintptr_t)d_out_state | (uintptr_t)d_out_conv) & 15)) return AVMP_EINVAL;
     c->launches += 1;
-    return cu(launch_ssm(c->g, false, layer, d_reqs, n, d_out_state, d_out_conv, L(c, stream)));
+    return cu(launch_ssm(c->g, false, layer, 1, d_reqs, n, d_out_state, 0, d_out_conv, 0, L(c, stream)));
 }
 
 int avmp_scatter_ssm(avmp_ctx *c, uint32_t layer, const uint32_t *d_reqs, uint32_t n, const void *d_in_state,
@@ -279,8 +279,37 @@ int avmp_scatter_ssm(avmp_ctx *c, uint32_t layer, const uint32_t *d_reqs, uint32
     if (n == 0) return AVMP_OK;
     if (!d_reqs || !d_in_state || !d_in_conv || (((uintptr_t)d_in_state | (uintptr_t)d_in_conv) & 15)) return AVMP_EINVAL;
     c->launches += 1;
-    return cu(launch_ssm(c->g, true, layer, d_reqs, n, const_cast<void *>(d_in_state),
-                         const_cast<void *>(d_in_conv), L(c, stream)));
+    return cu(launch_ssm(c->g, true, layer, 1, d_reqs, n, const_cast<void *>(d_in_state), 0,
+                         const_cast<void *>(d_in_conv), 0, L(c, stream)));
+}
+
+int avmp_gather_kv_layers(avmp_ctx *c, uint32_t first_layer, uint32_t n_layers, const uint32_t *d_reqs, uint32_t n,
+                          void *d_out_k, void *d_out_v, uint64_t layer_stride_bytes, uint64_t cap_tokens,
+                          uint32_t *d_cu, void *stream)
+{
+    if (!c || n_layers == 0 || (uint64_t)first_layer + n_layers > c->spec.n_attn_layers) return AVMP_EINVAL;
+    if (n > c->opt.max_requests || !d_cu) return AVMP_EINVAL;
+    if (n && (!d_reqs || !d_out_k || !d_out_v)) return AVMP_EINVAL;
+    if (((uintptr_t)d_out_k | (uintptr_t)d_out_v | layer_stride_bytes) & 15) return AVMP_EINVAL;
+    if (n_layers > 1 && layer_stride_bytes < cap_tokens * c->lay.kv_row_bytes) return AVMP_EINVAL;
+    c->launches += 2;
+    return cu(launch_kv(c->g, false, first_layer, n_layers, d_reqs, nullptr, n, d_out_k, d_out_v, layer_stride_bytes,
+                        cap_tokens, d_cu, L(c, stream)));
+}
+
+int avmp_gather_ssm_layers(avmp_ctx *c, uint32_t first_layer, uint32_t n_layers, const uint32_t *d_reqs, uint32_t n,
+                           void *d_out_state, uint64_t state_layer_stride_bytes, void *d_out_conv,
+                           uint64_t conv_layer_stride_bytes, void *stream)
+{
+    if (!c || n_layers == 0 || (uint64_t)first_layer + n_layers > c->spec.n_ssm_layers) return AVMP_EINVAL;
+    if (n == 0) return AVMP_OK;
+    if (!d_reqs || !d_out_state || !d_out_conv) return AVMP_EINVAL;
+    if (((uintptr_t)d_out_state | (uintptr_t)d_out_conv | state_layer_stride_bytes | conv_layer_stride_bytes) & 15) return AVMP_EINVAL;
+    if (n_layers > 1 && (state_layer_stride_bytes < (uint64_t)n * c->lay.ssm_state_bytes ||
+                         conv_layer_stride_bytes < (uint64_t)n * c->lay.ssm_conv_bytes)) return AVMP_EINVAL;
+    c->launches += 1;
+    return cu(launch_ssm(c->g, false, first_layer, n_layers, d_reqs, n, d_out_state, state_layer_stride_bytes,
+                         d_out_conv, conv_layer_stride_bytes, L(c, stream)));
 }
 
 int avmp_get_stats(avmp_ctx *c, avmp_stats *h_out, void *stream)

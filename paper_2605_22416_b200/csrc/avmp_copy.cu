@@ -55,20 +55,25 @@ struct Piece {
 };
 
 // ------------------------------- piece enumerators ------------------------------------
-// a12: SSM block <-> (state row, conv row) of the batch buffers.
+// a12: SSM block <-> (state row, conv row) of the batch buffers, for n_layers consecutive
+// layers (layer-major piece order; layer l's buffers start l * stride bytes further on).
 template <bool SCATTER>
 struct SsmPieces {
-    uint32_t layer, n, ps, per;
+    uint32_t layer0, n_layers, n, ps, per;
     const uint32_t *reqs;
     uint8_t *buf_state, *buf_conv;
-    __device__ unsigned long long total(const Geom &) const { return (unsigned long long)n * per; }
+    unsigned long long state_stride, conv_stride;
+    __device__ unsigned long long total(const Geom &) const { return (unsigned long long)n_layers * n * per; }
     __device__ Piece get(const Geom &g, unsigned long long it) const
     {
-        const uint32_t k = (uint32_t)(it / per), c = (uint32_t)(it % per);
+        const unsigned long long per_layer = (unsigned long long)n * per;
+        const uint32_t dl = (uint32_t)(it / per_layer);
+        const uint32_t rem = (uint32_t)(it % per_layer);
+        const uint32_t k = rem / per, c = rem % per;
         const uint32_t r = reqs[k];
         uint32_t slot = kInvalid;
         if (r < g.R && g.r_state[r] == AVMP_REQ_LIVE) {
-            const uint32_t h = g.r_ssm[(unsigned long long)r * g.ns + layer];
+            const uint32_t h = g.r_ssm[(unsigned long long)r * g.ns + layer0 + dl];
             if (h != kInvalid) slot = g.VT[1][h & 0x7FFFFFFFu];
         }
         if (slot == kInvalid) {
@@ -80,11 +85,11 @@ struct SsmPieces {
         uint32_t bytes;
         if (c < ps) {
             const unsigned long long o = (unsigned long long)c * kStage;
-            p = blk + o; b = buf_state + (unsigned long long)k * g.state_bytes + o;
+            p = blk + o; b = buf_state + dl * state_stride + (unsigned long long)k * g.state_bytes + o;
             bytes = (uint32_t)min((unsigned long long)kStage, g.state_bytes - o);
         } else {
             const unsigned long long o = (unsigned long long)(c - ps) * kStage;
-            p = blk + g.state_bytes + o; b = buf_conv + (unsigned long long)k * g.conv_bytes + o;
+            p = blk + g.state_bytes + o; b = buf_conv + dl * conv_stride + (unsigned long long)k * g.conv_bytes + o;
             bytes = (uint32_t)min((unsigned long long)kStage, g.conv_bytes - o);
         }
         return SCATTER ? Piece{b, p, bytes} : Piece{p, b, bytes};
@@ -117,19 +122,21 @@ struct RelocPieces {
 // (K slices, then V slices).
 template <bool SCATTER>
 struct KvPieces {
-    uint32_t layer, n, subs;
+    uint32_t layer0, n_layers, n, subs;
     const uint32_t *reqs, *tok_start;
     uint8_t *buf_k, *buf_v;
-    unsigned long long cap_tokens;
-    __device__ unsigned long long total(const Geom &g) const { return g.st->g_total_items; }
+    unsigned long long cap_tokens, layer_stride;
+    __device__ unsigned long long total(const Geom &g) const { return (unsigned long long)n_layers * g.st->g_total_items; }
     __device__ Piece get(const Geom &g, unsigned long long it64) const
     {
-        const uint32_t it = (uint32_t)it64;
+        const uint32_t per_layer = g.st->g_total_items;
+        const uint32_t dl = (uint32_t)(it64 / per_layer);
+        const uint32_t it = (uint32_t)(it64 % per_layer);
         const uint32_t k = find_owner(g.g_cu_items, 0u, n, 0u, it);
         const uint32_t rel = it - g.g_cu_items[k];
         const uint32_t row0 = g.g_cu_rows[k], rows = g.g_cu_rows[k + 1] - row0;
         if (!SCATTER && (unsigned long long)row0 + rows > cap_tokens) {
-            if (rel == 0) record_error(g.st, AVMP_DEV_OUT_OVERFLOW);
+            if (rel == 0 && dl == 0) record_error(g.st, AVMP_DEV_OUT_OVERFLOW);
             return Piece{nullptr, nullptr, 0};
         }
         const uint32_t T = g.T, row = (uint32_t)g.row_bytes, half = subs >> 1;
@@ -144,10 +151,10 @@ struct KvPieces {
         const uint32_t r = reqs[k];
         const uint32_t h = g.r_chain[(unsigned long long)r * g.max_pages + page];
         const uint32_t slot = g.VT[0][h & 0x7FFFFFFFu];
-        uint8_t *p = g.arena + (unsigned long long)slot * g.U[0] + (unsigned long long)layer * g.kv_layer_bytes +
+        uint8_t *p = g.arena + (unsigned long long)slot * g.U[0] + (unsigned long long)(layer0 + dl) * g.kv_layer_bytes +
                      (unsigned long long)part * T * row + b_lo;
         // byte b of the page part is byte (b - (t0 - page*T)*row) of the request's rows
-        uint8_t *b = (part ? buf_v : buf_k) +
+        uint8_t *b = (part ? buf_v : buf_k) + dl * layer_stride +
                      ((unsigned long long)row0 * row + (unsigned long long)page * T * row + b_lo -
                       (unsigned long long)t0 * row);
         return SCATTER ? Piece{b, p, b_hi - b_lo} : Piece{p, b, b_hi - b_lo};
@@ -211,11 +218,50 @@ __device__ __forceinline__ void bulk_wait_all()
 }
 
 // ------------------------------- the two skeletons --------------------------------------
+// Lane 0 of every warp drives the warp's ring; lanes 1..31 look up the next 31 pieces in
+// parallel (a lookup is a chain of three or four dependent table reads, far too slow to
+// sit on the issuing lane's path) and hand them over through shared memory, one batch ahead.
+struct Ring {
+    uint32_t buf0, bar0;
+    uint32_t n_loaded, n_stored;     // pieces issued as loads / as stores so far
+    uint8_t *dst[kStages];
+    uint32_t bytes[kStages];
+    bool failed;
+
+    // wait for the oldest load, then send its stage on its way to global memory
+    __device__ __forceinline__ void retire_one()
+    {
+        const uint32_t s = n_stored % kStages, parity = (n_stored / kStages) & 1u;
+        uint32_t spins = 0;
+        while (!mbar_try_wait(bar0 + 8u * s, parity))
+            if (++spins > kSpinLimit) { failed = true; return; }
+        bulk_s2g(dst[s], buf0 + s * kStage, bytes[s]);
+        ++n_stored;
+    }
+    __device__ __forceinline__ void push(const Piece &p)
+    {
+        if (n_loaded - n_stored == (uint32_t)kStages) retire_one();
+        if (failed) return;
+        const uint32_t s = n_loaded % kStages;
+        // the stage's previous occupant was piece n_loaded - kStages; its store (one bulk group per
+        // piece, in order) must have finished reading the buffer.  Only younger groups may pend.
+        if (n_loaded >= (uint32_t)kStages) wait_stage_free(n_stored - 1u - (n_loaded - (uint32_t)kStages));
+        dst[s] = p.dst;
+        bytes[s] = p.bytes;
+        mbar_expect_tx(bar0 + 8u * s, p.bytes);
+        bulk_g2s(buf0 + s * kStage, p.src, p.bytes, bar0 + 8u * s);
+        ++n_loaded;
+    }
+};
+
+constexpr int kBatch = 31;   // pieces looked up per hand-over (lanes 1..31)
+
 template <class F>
 __global__ void __launch_bounds__(kBulkThreads, kBulkCtasPerSm) stream_bulk_kernel(const Geom g, const F f)
 {
-    extern __shared__ __align__(1024) uint8_t ring[];
+    extern __shared__ __align__(1024) uint8_t ring_mem[];
     __shared__ __align__(8) unsigned long long bars[kBulkWarps * kStages];
+    __shared__ Piece handover[kBulkWarps][2][kBatch];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const unsigned long long total = f.total(g);
@@ -223,46 +269,47 @@ __global__ void __launch_bounds__(kBulkThreads, kBulkCtasPerSm) stream_bulk_kern
         for (int s = 0; s < kStages; ++s) mbar_init(smem_u32(&bars[warp * kStages + s]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
-    if (lane != 0) return;               // one lane drives its warp's ring
 
-    const uint32_t buf0 = smem_u32(ring) + (uint32_t)warp * kStages * kStage;
-    const uint32_t bar0 = smem_u32(&bars[warp * kStages]);
-    Piece pc[kStages];                   // piece sitting in each stage
-    uint32_t n_loaded = 0, n_stored = 0; // pieces issued as loads / as stores so far
-    bool drained = false, failed = false;
-    // warp w of CTA c takes pieces (w * grid + c) + j * (grid * warps), j = 0, 1, ...
+    // warp w of CTA c takes pieces (w * grid + c) + j * (grid * warps), j = 0, 1, ...: at any moment
+    // the pieces in flight across the grid form one dense window of the list
     const unsigned long long first = (unsigned long long)warp * gridDim.x + blockIdx.x;
     const unsigned long long stride = (unsigned long long)gridDim.x * kBulkWarps;
-    unsigned long long n_taken = 0;
+    if (first >= total) return;
+    const unsigned long long mine = (total - first + stride - 1) / stride;       // pieces of this warp
+    const uint32_t n_batches = (uint32_t)((mine + kBatch - 1) / kBatch);
 
-    // Each loop turn: top up the ring with loads, then retire the oldest stage with a store.
-    while (true) {
-        while (!drained && n_loaded - n_stored < (uint32_t)kStages) {
-            const unsigned long long it = first + n_taken * stride;
-            ++n_taken;
-            if (it >= total) { drained = true; break; }
-            const Piece p = f.get(g, it);
-            if (p.bytes == 0) continue;
-            const uint32_t s = n_loaded % kStages;
-            // the stage's previous occupant was piece n_loaded - kStages; its store (one bulk group
-            // per piece, in order) must have finished reading the buffer.  Only younger groups may pend.
-            if (n_loaded >= (uint32_t)kStages) wait_stage_free(n_stored - 1u - (n_loaded - (uint32_t)kStages));
-            pc[s] = p;
-            mbar_expect_tx(bar0 + 8u * s, p.bytes);
-            bulk_g2s(buf0 + s * kStage, p.src, p.bytes, bar0 + 8u * s);
-            ++n_loaded;
+    Ring ring;
+    ring.buf0 = smem_u32(ring_mem) + (uint32_t)warp * kStages * kStage;
+    ring.bar0 = smem_u32(&bars[warp * kStages]);
+    ring.n_loaded = ring.n_stored = 0;
+    ring.failed = false;
+
+    auto lookup = [&](uint32_t batch) {            // lanes 1..31
+        const unsigned long long j = (unsigned long long)batch * kBatch + (lane - 1);
+        Piece p{nullptr, nullptr, 0};
+        if (j < mine) p = f.get(g, first + j * stride);
+        handover[warp][batch & 1][lane - 1] = p;
+    };
+    if (lane != 0) lookup(0);
+    __syncwarp();
+    for (uint32_t b = 0; b < n_batches; ++b) {
+        if (lane != 0) {
+            if (b + 1 < n_batches) lookup(b + 1);
+        } else {
+            const unsigned long long left = mine - (unsigned long long)b * kBatch;
+            const int cnt = left < (unsigned long long)kBatch ? (int)left : kBatch;
+            for (int i = 0; i < cnt && !ring.failed; ++i) {
+                const Piece p = handover[warp][b & 1][i];
+                if (p.bytes) ring.push(p);
+            }
         }
-        if (n_stored == n_loaded) break;
-        const uint32_t s = n_stored % kStages, parity = (n_stored / kStages) & 1u;
-        uint32_t spins = 0;
-        while (!mbar_try_wait(bar0 + 8u * s, parity))
-            if (++spins > kSpinLimit) { failed = true; break; }
-        if (failed) break;
-        bulk_s2g(pc[s].dst, buf0 + s * kStage, pc[s].bytes);
-        ++n_stored;
+        __syncwarp();
     }
-    if (failed) record_error(g.st, AVMP_DEV_TIMEOUT);
-    bulk_wait_all();
+    if (lane == 0) {
+        while (!ring.failed && ring.n_stored < ring.n_loaded) ring.retire_one();
+        if (ring.failed) record_error(g.st, AVMP_DEV_TIMEOUT);
+        bulk_wait_all();
+    }
 }
 
 template <class F>
@@ -383,8 +430,8 @@ cudaError_t launch_translate(const Geom &g, const uint32_t *h, uint32_t n, uint3
     return cudaGetLastError();
 }
 
-cudaError_t launch_kv(const Geom &g, bool scatter, uint32_t layer, const uint32_t *reqs,
-                      const uint32_t *tok_start, uint32_t n, void *k, void *v,
+cudaError_t launch_kv(const Geom &g, bool scatter, uint32_t layer0, uint32_t n_layers, const uint32_t *reqs,
+                      const uint32_t *tok_start, uint32_t n, void *k, void *v, unsigned long long layer_stride,
                       unsigned long long cap_tokens, uint32_t *cu_out, const Launch &l)
 {
     const unsigned long long part = (unsigned long long)g.T * g.row_bytes;     // K (or V) bytes of a page
@@ -392,20 +439,22 @@ cudaError_t launch_kv(const Geom &g, bool scatter, uint32_t layer, const uint32_
     kv_plan_kernel<<<1, kStepThreads, 0, l.stream>>>(g, reqs, tok_start, n, subs, cu_out);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    const bool bulk_ok = mult16(g.row_bytes) && mult16(g.U[0]) && mult16(g.kv_layer_bytes);
+    const bool bulk_ok = mult16(g.row_bytes) && mult16(g.U[0]) && mult16(g.kv_layer_bytes) && mult16(layer_stride);
     if (scatter)
-        return launch_stream(g, KvPieces<true>{layer, n, subs, reqs, tok_start, (uint8_t *)k, (uint8_t *)v, cap_tokens}, bulk_ok, l);
-    return launch_stream(g, KvPieces<false>{layer, n, subs, reqs, tok_start, (uint8_t *)k, (uint8_t *)v, cap_tokens}, bulk_ok, l);
+        return launch_stream(g, KvPieces<true>{layer0, n_layers, n, subs, reqs, tok_start, (uint8_t *)k, (uint8_t *)v, cap_tokens, layer_stride}, bulk_ok, l);
+    return launch_stream(g, KvPieces<false>{layer0, n_layers, n, subs, reqs, tok_start, (uint8_t *)k, (uint8_t *)v, cap_tokens, layer_stride}, bulk_ok, l);
 }
 
-cudaError_t launch_ssm(const Geom &g, bool scatter, uint32_t layer, const uint32_t *reqs, uint32_t n,
-                       void *state, void *conv, const Launch &l)
+cudaError_t launch_ssm(const Geom &g, bool scatter, uint32_t layer0, uint32_t n_layers, const uint32_t *reqs, uint32_t n,
+                       void *state, unsigned long long state_stride, void *conv, unsigned long long conv_stride,
+                       const Launch &l)
 {
     const uint32_t ps = (uint32_t)((g.state_bytes + kStage - 1) / kStage), pc = (uint32_t)((g.conv_bytes + kStage - 1) / kStage);
-    const bool bulk_ok = mult16(g.state_bytes) && mult16(g.conv_bytes) && mult16(g.U[1]) && mult16(g.P_al);
+    const bool bulk_ok = mult16(g.state_bytes) && mult16(g.conv_bytes) && mult16(g.U[1]) && mult16(g.P_al) &&
+                         mult16(state_stride) && mult16(conv_stride);
     if (scatter)
-        return launch_stream(g, SsmPieces<true>{layer, n, ps, ps + pc, reqs, (uint8_t *)state, (uint8_t *)conv}, bulk_ok, l);
-    return launch_stream(g, SsmPieces<false>{layer, n, ps, ps + pc, reqs, (uint8_t *)state, (uint8_t *)conv}, bulk_ok, l);
+        return launch_stream(g, SsmPieces<true>{layer0, n_layers, n, ps, ps + pc, reqs, (uint8_t *)state, (uint8_t *)conv, state_stride, conv_stride}, bulk_ok, l);
+    return launch_stream(g, SsmPieces<false>{layer0, n_layers, n, ps, ps + pc, reqs, (uint8_t *)state, (uint8_t *)conv, state_stride, conv_stride}, bulk_ok, l);
 }
 
 }  // namespace avmp

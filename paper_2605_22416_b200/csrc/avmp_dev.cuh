@@ -120,11 +120,12 @@ cudaError_t launch_step(const Geom &g, const avmp_op *d_ops, uint32_t n_ops, uin
 cudaError_t launch_relocate(const Geom &g, const Launch &l);
 cudaError_t launch_translate(const Geom &g, const uint32_t *h, uint32_t n, uint32_t *pool,
                              unsigned long long *off, unsigned long long *aoff, const Launch &l);
-cudaError_t launch_kv(const Geom &g, bool scatter, uint32_t layer, const uint32_t *reqs,
-                      const uint32_t *tok_start, uint32_t n, void *k, void *v,
+cudaError_t launch_kv(const Geom &g, bool scatter, uint32_t layer0, uint32_t n_layers, const uint32_t *reqs,
+                      const uint32_t *tok_start, uint32_t n, void *k, void *v, unsigned long long layer_stride,
                       unsigned long long cap_tokens, uint32_t *cu_out, const Launch &l);
-cudaError_t launch_ssm(const Geom &g, bool scatter, uint32_t layer, const uint32_t *reqs, uint32_t n,
-                       void *state, void *conv, const Launch &l);
+cudaError_t launch_ssm(const Geom &g, bool scatter, uint32_t layer0, uint32_t n_layers, const uint32_t *reqs, uint32_t n,
+                       void *state, unsigned long long state_stride, void *conv, unsigned long long conv_stride,
+                       const Launch &l);
 
 }  // namespace avmp
 

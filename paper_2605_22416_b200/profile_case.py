@@ -1,7 +1,8 @@
 """Small, self-contained launches of each kernel for profiling (a few GB on the device,
 a handful of launches): `python -m paper_2605_22416_b200.profile_case <case>`.
 
-Cases: ssm_gather, kv_gather, relocate, step.  Every case builds a context through the
+Cases: ssm_gather, kv_gather (one layer per launch), ssm_gather_fused, kv_gather_fused (several
+layers per launch), relocate, step.  Every case builds a context through the
 C ABI, brings it to a busy state with a few allocator steps and then launches the kernel
 of interest `--repeat` times on different layers, so every launch reads cold data.
 """
@@ -22,13 +23,49 @@ def _dev(a):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["ssm_gather", "kv_gather", "relocate", "step"])
+    ap.add_argument("case", choices=["ssm_gather", "kv_gather", "ssm_gather_fused", "kv_gather_fused", "relocate", "step"])
     ap.add_argument("--repeat", type=int, default=6)
     ap.add_argument("--pool-gib", type=float, default=3.0)
+    ap.add_argument("--layers", type=int, default=8, help="layers per launch in the fused cases")
     args = ap.parse_args()
     m = W.JAMBA_LIKE
     pool = int(args.pool_gib * W.GiB)
     ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    if args.case in ("ssm_gather_fused", "kv_gather_fused"):
+        kv = args.case == "kv_gather_fused"
+        nl = min(args.layers, m.n_attn_layers if kv else m.n_ssm_layers)
+        n_req, tokens = (48, 2048) if kv else (150, 64)
+        ctx = B.Context(m, pool, 0.3 if kv else 0.85, 128, max_requests=256, max_pages=256)
+        st = np.zeros(n_req, np.uint32)
+        ctx.step_host(W.make_ops(W.OP_ADMIT, np.arange(n_req), tokens), n_req, st)
+        assert (st == 0).all(), st
+        reqs = _dev(np.random.default_rng(0).permutation(n_req).astype(np.uint32))
+        if kv:
+            tot = n_req * tokens
+            cu = torch.zeros(n_req + 1, dtype=torch.int32, device="cuda")
+            ok = torch.empty((nl, tot, m.kv_row_bytes), dtype=torch.uint8, device="cuda")
+            ov = torch.empty((nl, tot, m.kv_row_bytes), dtype=torch.uint8, device="cuda")
+            nbytes = 2 * tot * 2 * m.kv_row_bytes * nl
+        else:
+            os_ = torch.empty((nl, n_req, m.state_bytes), dtype=torch.uint8, device="cuda")
+            oc = torch.empty((nl, n_req, m.conv_bytes), dtype=torch.uint8, device="cuda")
+            nbytes = 2 * n_req * (m.state_bytes + m.conv_bytes) * nl
+        for i in range(args.repeat):
+            first = (i * nl) % ((m.n_attn_layers if kv else m.n_ssm_layers) - nl + 1)
+            a, b = ev(), ev()
+            a.record()
+            if kv:
+                ctx.gather_kv_layers(first, nl, reqs, n_req, ok, ov, tot * m.kv_row_bytes, tot, cu)
+            else:
+                ctx.gather_ssm_layers(first, nl, reqs, n_req, os_, n_req * m.state_bytes, oc, n_req * m.conv_bytes)
+            b.record()
+            torch.cuda.synchronize()
+            print(f"{args.case} launch {i} ({nl} layers from {first}): {a.elapsed_time(b) * 1e3:.1f} us, "
+                  f"{nbytes / 1e6:.0f} MB, {nbytes / a.elapsed_time(b) / 1e6:.0f} GB/s")
+        print(ctx.stats())
+        ctx.close()
+        return
 
     if args.case in ("ssm_gather", "kv_gather", "step"):
         split = 0.85 if args.case != "kv_gather" else 0.3

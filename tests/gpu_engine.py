@@ -77,6 +77,25 @@ class GpuEngine:
         bad = self.ctx.stats()["error_count"] - before
         return st.cpu().numpy()[:n], cv.cpu().numpy()[:n], bad
 
+    def gather_kv_layers(self, first, n_layers, reqs, capacity_tokens):
+        r = np.ascontiguousarray(reqs, dtype=np.uint32)
+        row = self.model.kv_row_bytes
+        cap = max(capacity_tokens, 1)
+        out_k = torch.zeros((n_layers, cap, row), dtype=torch.uint8, device=self.dev)
+        out_v = torch.zeros((n_layers, cap, row), dtype=torch.uint8, device=self.dev)
+        cu = torch.zeros(len(r) + 1, dtype=torch.int32, device=self.dev)
+        self.ctx.gather_kv_layers(first, n_layers, self._dev(r), len(r), out_k, out_v, cap * row, capacity_tokens, cu)
+        return out_k.cpu().numpy(), out_v.cpu().numpy(), cu.cpu().numpy().view(np.uint32)
+
+    def gather_ssm_layers(self, first, n_layers, reqs):
+        r = np.ascontiguousarray(reqs, dtype=np.uint32)
+        n = max(len(r), 1)
+        st = torch.zeros((n_layers, n, self.model.state_bytes), dtype=torch.uint8, device=self.dev)
+        cv = torch.zeros((n_layers, n, self.model.conv_bytes), dtype=torch.uint8, device=self.dev)
+        self.ctx.gather_ssm_layers(first, n_layers, self._dev(r), len(r), st, n * self.model.state_bytes,
+                                   cv, n * self.model.conv_bytes)
+        return st.cpu().numpy(), cv.cpu().numpy()
+
     def scatter_kv(self, layer, reqs, tok_start, in_k, in_v) -> int:
         r = np.ascontiguousarray(reqs, dtype=np.uint32)
         before = self.ctx.stats()["error_count"]

@@ -198,6 +198,42 @@ def test_pr1_small_pool_relocations(env):
     assert s["relocated_blocks"] > 10 and s["n_rebalance"] > 5
 
 
+def test_multi_layer_gathers(env):
+    """avmp_gather_kv_layers / avmp_gather_ssm_layers: one launch for a range of layers gives,
+    layer by layer, the oracle's single-layer gathers (and the payload function's bytes)."""
+    w = W.config("pr1", pool_bytes=48 * W.MiB, concurrency=16, min_rebalance_interval_ops=50,
+                 migration_batch_size=6, n_requests=120)
+    g, o = _pair(env, w, with_store=True)
+    h = PayloadHarness(w, [g, o])              # payload on every layer
+    d = W.ClosedLoopDriver(w)
+
+    def step(ops):
+        so = o.step(ops)
+        assert np.array_equal(g.step(ops), so)
+        return so
+
+    W.record_trace(w, step, max_steps=260, driver=d, on_step=lambda d, a, b: h.apply_writes(d.writes))
+    assert g.stats()["n_rebalance"] > 0
+    run = d.running_slots.astype(np.uint32)
+    assert len(run) > 3
+    tot = int(d.len[run].sum())
+    m = w.model
+    for first, nl in ((0, m.n_attn_layers), (1, 2), (3, 1)):
+        gk, gv, gcu = g.gather_kv_layers(first, nl, run, tot)
+        for l in range(nl):
+            ok, ov, ocu, bad = o.gather_kv(first + l, run, tot)
+            assert bad == 0 and np.array_equal(gcu, ocu)
+            assert np.array_equal(gk[l][:tot], ok) and np.array_equal(gv[l][:tot], ov)
+            ek, ev_, _ = h.expected_kv(first + l, d.uid[run], d.len[run])
+            assert np.array_equal(gk[l][:tot], ek) and np.array_equal(gv[l][:tot], ev_)
+    for first, nl in ((0, m.n_ssm_layers), (5, 3), (11, 1)):
+        gs, gc = g.gather_ssm_layers(first, nl, run)
+        for l in range(nl):
+            os_, oc, bad = o.gather_ssm(first + l, run)
+            assert bad == 0 and np.array_equal(gs[l], os_) and np.array_equal(gc[l], oc)
+    assert g.stats()["error_code"] == 0
+
+
 @pytest.mark.parametrize("name,steps,over", [
     ("short_uniform", 1200, {}),
     ("short_uniform", 500, dict(seed=1)),
