@@ -23,7 +23,7 @@ struct Carve {
 
 // Offsets of every table inside the workspace, in one place so that size and carving agree.
 struct WsLayout {
-    size_t state, S[2], W[2], VT[2], OW[2], r_state, r_len, r_npages, r_chain, r_ssm, mark;
+    size_t state, S[2], W[2], VT[2], OW[2], r_state, r_len, r_npages, r_chain, r_ssm;
     size_t reloc_src, reloc_dst, g_cu_items, g_cu_rows, stage_ops, stage_status, total;
 };
 
@@ -40,7 +40,6 @@ WsLayout ws_layout(const avmp_layout &lay, const avmp_model_spec &spec, const av
     w.r_state = c.take(R * 4); w.r_len = c.take(R * 4); w.r_npages = c.take(R * 4);
     w.r_chain = c.take(R * (size_t)opt.max_pages_per_request * 4);
     w.r_ssm = c.take(R * (size_t)spec.n_ssm_layers * 4);
-    w.mark = c.take(R * 4);
     const size_t maxv = (size_t)(lay.vid_space[0] > lay.vid_space[1] ? lay.vid_space[0] : lay.vid_space[1]);
     w.reloc_src = c.take(maxv * 4); w.reloc_dst = c.take(maxv * 4);
     w.g_cu_items = c.take((R + 1) * 4); w.g_cu_rows = c.take((R + 1) * 4);
@@ -168,7 +167,7 @@ int avmp_create(avmp_ctx **out, const avmp_model_spec *spec, void *d_arena, uint
     }
     g.r_state = reinterpret_cast<uint32_t *>(base + w.r_state); g.r_len = reinterpret_cast<uint32_t *>(base + w.r_len);
     g.r_npages = reinterpret_cast<uint32_t *>(base + w.r_npages); g.r_chain = reinterpret_cast<uint32_t *>(base + w.r_chain);
-    g.r_ssm = reinterpret_cast<uint32_t *>(base + w.r_ssm); g.mark = reinterpret_cast<uint32_t *>(base + w.mark);
+    g.r_ssm = reinterpret_cast<uint32_t *>(base + w.r_ssm);
     g.reloc_src = reinterpret_cast<uint32_t *>(base + w.reloc_src); g.reloc_dst = reinterpret_cast<uint32_t *>(base + w.reloc_dst);
     g.g_cu_items = reinterpret_cast<uint32_t *>(base + w.g_cu_items); g.g_cu_rows = reinterpret_cast<uint32_t *>(base + w.g_cu_rows);
     c->d_stage_ops = reinterpret_cast<avmp_op *>(base + w.stage_ops);

@@ -264,11 +264,12 @@ __global__ void __launch_bounds__(kBulkThreads, kBulkCtasPerSm) stream_bulk_kern
     __shared__ Piece handover[kBulkWarps][2][kBatch];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const unsigned long long total = f.total(g);
     if (lane == 0)
         for (int s = 0; s < kStages; ++s) mbar_init(smem_u32(&bars[warp * kStages + s]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    pdl_prologue();
     __syncthreads();
+    const unsigned long long total = f.total(g);
 
     // warp w of CTA c takes pieces (w * grid + c) + j * (grid * warps), j = 0, 1, ...: at any moment
     // the pieces in flight across the grid form one dense window of the list
@@ -316,6 +317,7 @@ template <class F>
 __global__ void __launch_bounds__(kGenThreads) stream_generic_kernel(const Geom g, const F f)
 {
     const int lane = threadIdx.x & 31;
+    pdl_prologue();
     const unsigned long long total = f.total(g);
     const unsigned long long nw = (unsigned long long)gridDim.x * (kGenThreads / 32);
     for (unsigned long long it = (unsigned long long)(threadIdx.x >> 5) * gridDim.x + blockIdx.x; it < total; it += nw) {
@@ -344,11 +346,9 @@ cudaError_t launch_stream(const Geom &g, const F &f, bool bulk_ok, const Launch 
             if (e != cudaSuccess) return e;
             attr_set[l.device & 63] = true;
         }
-        stream_bulk_kernel<F><<<l.n_sms * kBulkCtasPerSm, kBulkThreads, kBulkSmem, l.stream>>>(g, f);
-    } else {
-        stream_generic_kernel<F><<<l.n_sms * kGenCtasPerSm, kGenThreads, 0, l.stream>>>(g, f);
+        return launch_pdl(stream_bulk_kernel<F>, dim3(l.n_sms * kBulkCtasPerSm), dim3(kBulkThreads), kBulkSmem, l.stream, g, f);
     }
-    return cudaGetLastError();
+    return launch_pdl(stream_generic_kernel<F>, dim3(l.n_sms * kGenCtasPerSm), dim3(kGenThreads), 0, l.stream, g, f);
 }
 
 inline bool mult16(unsigned long long x) { return (x & 15ull) == 0; }
@@ -358,6 +358,7 @@ __global__ void translate_kernel(const Geom g, const uint32_t *__restrict__ h, u
                                  uint32_t *__restrict__ pool, unsigned long long *__restrict__ off,
                                  unsigned long long *__restrict__ aoff)
 {
+    pdl_prologue();
     for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
         const uint32_t hv = h[i], p = hv >> 31, vid = hv & 0x7FFFFFFFu;
         uint32_t slot = kInvalid;
@@ -381,6 +382,7 @@ kv_plan_kernel(const Geom g, const uint32_t *__restrict__ reqs, const uint32_t *
     __shared__ unsigned long long tmp[32];
     unsigned long long run_rows = 0, run_items = 0, tot;
     const int tid = threadIdx.x;
+    pdl_prologue();
     for (uint32_t b = 0; b < n; b += kStepThreads) {
         const uint32_t k = b + tid;
         uint32_t rows = 0, items = 0;
@@ -426,8 +428,7 @@ cudaError_t launch_translate(const Geom &g, const uint32_t *h, uint32_t n, uint3
                              unsigned long long *off, unsigned long long *aoff, const Launch &l)
 {
     const int blocks = (int)min((unsigned long long)l.n_sms * 4, ((unsigned long long)n + 255) / 256);
-    translate_kernel<<<blocks, 256, 0, l.stream>>>(g, h, n, pool, off, aoff);
-    return cudaGetLastError();
+    return launch_pdl(translate_kernel, dim3(blocks), dim3(256), 0, l.stream, g, h, n, pool, off, aoff);
 }
 
 cudaError_t launch_kv(const Geom &g, bool scatter, uint32_t layer0, uint32_t n_layers, const uint32_t *reqs,
@@ -436,8 +437,7 @@ cudaError_t launch_kv(const Geom &g, bool scatter, uint32_t layer0, uint32_t n_l
 {
     const unsigned long long part = (unsigned long long)g.T * g.row_bytes;     // K (or V) bytes of a page
     const uint32_t subs = 2u * (uint32_t)((part + kStage - 1) / kStage);
-    kv_plan_kernel<<<1, kStepThreads, 0, l.stream>>>(g, reqs, tok_start, n, subs, cu_out);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_pdl(kv_plan_kernel, dim3(1), dim3(kStepThreads), 0, l.stream, g, reqs, tok_start, n, subs, cu_out);
     if (e != cudaSuccess) return e;
     const bool bulk_ok = mult16(g.row_bytes) && mult16(g.U[0]) && mult16(g.kv_layer_bytes) && mult16(layer_stride);
     if (scatter)

@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 #include "avmp.h"
 
 namespace avmp {
@@ -34,7 +36,7 @@ struct Geom {
     uint8_t *arena;
     DevState *st;
     uint32_t *S[2], *W[2], *VT[2], *OW[2];
-    uint32_t *r_state, *r_len, *r_npages, *r_chain, *r_ssm, *mark;
+    uint32_t *r_state, *r_len, *r_npages, *r_chain, *r_ssm;
     uint32_t *reloc_src, *reloc_dst;
     uint32_t *g_cu_items, *g_cu_rows;   // gather scratch, R + 1 entries each
 };
@@ -106,6 +108,35 @@ __device__ __forceinline__ uint32_t find_owner(const uint32_t *a, uint32_t lo, u
         if (a[mid] - base <= u) lo = mid; else hi = mid;
     }
     return lo;
+}
+
+// ---- programmatic dependent launch ------------------------------------------------------
+// Every kernel of the library starts with pdl_prologue(): it lets the next kernel in the stream
+// be scheduled at once (its CTAs become resident as resources free up and its launch latency is
+// hidden), then waits until everything before it in the stream has completed and is visible.
+// No global memory is touched before the wait, so stream order is preserved exactly; launched
+// without the attribute the two instructions do nothing.
+__device__ __forceinline__ void pdl_prologue()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+template <class... KArgs, class... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                              Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
 // Host-side launch wrappers (defined next to their kernels).

@@ -6,6 +6,7 @@
 // slots.  Inside a run the sequential result has a closed form:
 //   * free run  -- an exclusive prefix sum of the units each op releases gives the stack
 //                  position of every pushed slot and id;
+//   (same-slot repeats inside a window are found with a shared-memory hash of the slots)
 //   * alloc run -- an exclusive prefix sum of the demands gives the stack entries every op
 //                  pops, as long as every op before it fits.  The first op whose inclusive
 //                  demand exceeds the free count is the first sequential failure: everything
@@ -37,9 +38,12 @@ struct Scalars {
     unsigned long long mig_waste;
 };
 
+constexpr uint32_t kHash = 2 * NT;     // open-addressing table for same-slot detection
+
 struct Shared {
     uint32_t excl_k[NT + 1], excl_s[NT + 1];
     uint32_t req[NT], base[NT];
+    uint32_t hkey[kHash], hval[kHash];
     uint8_t dir[NT];
     unsigned long long tmp64[32];
     uint32_t tmp32[32];
@@ -187,6 +191,7 @@ step_kernel(const Geom g, const avmp_op *__restrict__ ops, const uint32_t n_ops,
     Scalars &sc = sh.sc;
     const int tid = threadIdx.x;
     DevState *ds = g.st;
+    pdl_prologue();
 
     if (tid == 0) {
         sc.last = ds->last_rebalance_op; sc.n_oom = ds->n_oom; sc.n_ce = ds->n_capacity_error;
@@ -225,16 +230,31 @@ step_kernel(const Geom g, const avmp_op *__restrict__ ops, const uint32_t n_ops,
         }
         sh.dir[tid] = dir;
         sh.req[tid] = req;
-        // ---- same-slot dependencies inside the window ----
-        if (dir >= DIR_ALLOC) atomicMin(&g.mark[req], (uint32_t)tid);
+        // request record, fetched now so the loads overlap the bookkeeping below; ops whose slot
+        // appears earlier in the window read it again when their run starts
+        uint32_t pf_state = 0, pf_len = 0, pf_np = 0;
+        if (dir >= DIR_ALLOC) { pf_state = g.r_state[req]; pf_len = g.r_len[req]; pf_np = g.r_npages[req]; }
+        // ---- same-slot dependencies inside the window: shared-memory hash, slot -> first op ----
+        sh.hkey[tid] = INF; sh.hkey[tid + NT] = INF;
+        sh.hval[tid] = INF; sh.hval[tid + NT] = INF;
         __syncthreads();
-        const bool dupflag = dir >= DIR_ALLOC && g.mark[req] != (uint32_t)tid;
+        uint32_t hs = 0;
+        if (dir >= DIR_ALLOC) {
+            hs = (req * 2654435761u) >> 21;                      // 11 bits
+            while (true) {
+                const uint32_t old = atomicCAS(&sh.hkey[hs], INF, req);
+                if (old == INF || old == req) break;
+                hs = (hs + 1u) & (kHash - 1u);
+            }
+            atomicMin(&sh.hval[hs], (uint32_t)tid);
+        }
+        __syncthreads();
+        const bool dupflag = dir >= DIR_ALLOC && sh.hval[hs] != (uint32_t)tid;
         const int any_dup = __syncthreads_or(dupflag);
         int prev_same = -1;
         if (any_dup && dupflag)
             for (int j = tid - 1; j >= 0; --j)
                 if (sh.dir[j] >= DIR_ALLOC && sh.req[j] == req) { prev_same = j; break; }
-        if (dir >= DIR_ALLOC) g.mark[req] = INF;
 
         uint32_t cur = 0;
         while (cur < wn) {
@@ -253,10 +273,11 @@ step_kernel(const Geom g, const avmp_op *__restrict__ ops, const uint32_t n_ops,
                 bool valid = false;
                 const bool keep = (flags & AVMP_FLAG_KEEP_KV) != 0;
                 if (in_run) {
-                    rstate = g.r_state[req];
+                    const bool fresh = prev_same < 0;
+                    rstate = fresh ? pf_state : g.r_state[req];
                     if (rstate == AVMP_REQ_LIVE || rstate == AVMP_REQ_KV_ONLY) {
                         valid = true;
-                        nk = keep ? 0u : g.r_npages[req];
+                        nk = keep ? 0u : (fresh ? pf_np : g.r_npages[req]);
                         nsu = rstate == AVMP_REQ_LIVE ? g.ns : 0u;
                         st = AVMP_ST_OK;
                     } else st = AVMP_ST_BAD_REQ;
@@ -304,7 +325,8 @@ step_kernel(const Geom g, const avmp_op *__restrict__ ops, const uint32_t n_ops,
                 uint32_t nk = 0, nsu = 0, new_len = 0;
                 bool valid = false;
                 if (in_run) {
-                    const uint32_t rstate = g.r_state[req];
+                    const bool fresh = prev_same < 0;
+                    const uint32_t rstate = fresh ? pf_state : g.r_state[req];
                     bool ok_state;
                     if (kind == AVMP_OP_ADMIT)
                         ok_state = (flags & AVMP_FLAG_RESUME) ? rstate == AVMP_REQ_KV_ONLY : rstate == AVMP_REQ_EMPTY;
@@ -312,9 +334,9 @@ step_kernel(const Geom g, const avmp_op *__restrict__ ops, const uint32_t n_ops,
                         ok_state = rstate == AVMP_REQ_LIVE;
                     if (!ok_state) st = AVMP_ST_BAD_REQ;
                     else {
-                        const unsigned long long nl = (unsigned long long)g.r_len[req] + tokens;
+                        const unsigned long long nl = (unsigned long long)(fresh ? pf_len : g.r_len[req]) + tokens;
                         const unsigned long long pages = (nl + g.T - 1ull) / g.T;
-                        const uint32_t have = g.r_npages[req];
+                        const uint32_t have = fresh ? pf_np : g.r_npages[req];
                         if (pages > g.max_pages || nl > 0xFFFFFFFFull) st = AVMP_ST_TOO_LONG;
                         else {
                             valid = true;
@@ -412,6 +434,7 @@ __global__ void init_kernel(const Geom g, const DevState init)
 {
     const unsigned long long gid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+    pdl_prologue();
     if (gid == 0) *g.st = init;
     for (int p = 0; p < 2; ++p) {
         const uint32_t V = g.V[p], cap = init.cap[p];
@@ -423,7 +446,7 @@ __global__ void init_kernel(const Geom g, const DevState init)
         }
     }
     for (unsigned long long i = gid; i < g.R; i += stride) {
-        g.r_state[i] = AVMP_REQ_EMPTY; g.r_len[i] = 0; g.r_npages[i] = 0; g.mark[i] = kInvalid;
+        g.r_state[i] = AVMP_REQ_EMPTY; g.r_len[i] = 0; g.r_npages[i] = 0;
     }
     for (unsigned long long i = gid; i < (unsigned long long)g.R * g.max_pages; i += stride) g.r_chain[i] = kInvalid;
     for (unsigned long long i = gid; i < (unsigned long long)g.R * g.ns; i += stride) g.r_ssm[i] = kInvalid;
@@ -433,15 +456,13 @@ __global__ void init_kernel(const Geom g, const DevState init)
 
 cudaError_t launch_init(const Geom &g, const DevState &init, cudaStream_t s)
 {
-    init_kernel<<<296, 512, 0, s>>>(g, init);
-    return cudaGetLastError();
+    return launch_pdl(init_kernel, dim3(296), dim3(512), 0, s, g, init);
 }
 
 cudaError_t launch_step(const Geom &g, const avmp_op *d_ops, uint32_t n_ops, uint32_t *d_status,
                         int first_round, cudaStream_t s)
 {
-    step_kernel<<<1, NT, 0, s>>>(g, d_ops, n_ops, d_status, first_round);
-    return cudaGetLastError();
+    return launch_pdl(step_kernel, dim3(1), dim3(NT), 0, s, g, d_ops, n_ops, d_status, first_round);
 }
 
 }  // namespace avmp

@@ -37,6 +37,8 @@ def main():
         nl = min(args.layers, m.n_attn_layers if kv else m.n_ssm_layers)
         n_req, tokens = (48, 2048) if kv else (150, 64)
         ctx = B.Context(m, pool, 0.3 if kv else 0.85, 128, max_requests=256, max_pages=256)
+        s0 = ctx.stats()
+        n_req = min(n_req, s0["cap_ssm"] // m.n_ssm_layers, s0["cap_kv"] // (tokens // 16))
         st = np.zeros(n_req, np.uint32)
         ctx.step_host(W.make_ops(W.OP_ADMIT, np.arange(n_req), tokens), n_req, st)
         assert (st == 0).all(), st
@@ -119,7 +121,7 @@ def main():
     # the whole store, then exhaust the SSM store: the migration cedes the top of the KV store
     # and must move the live pages it finds there.
     B_units = 4096
-    ctx = B.Context(m, pool, 0.3, B_units, max_requests=512, max_pages=256, min_rebalance_interval_ops=1)
+    ctx = B.Context(m, pool, 0.3, B_units, max_requests=512, max_pages=256)
     s0 = ctx.stats()
     n_req = min(400, s0["cap_ssm"] // m.n_ssm_layers)
     per = min(256, s0["cap_kv"] // n_req)
