@@ -351,6 +351,92 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
 
 
 # ---------------------------------------------------------------------------------------
+# micro-benchmarks reported beside the headline: one large migration, allocator rate vs batch
+# ---------------------------------------------------------------------------------------
+def migration_microbench(dev) -> dict:
+    """Fill the KV store, free every other request so live pages are striped over the whole
+    store, then exhaust the SSM store: one CapacityError cedes the top 16 384 KV pages and the
+    migration must move every live page it finds there (about 2 GB)."""
+    import torch
+    from paper_2605_22416_b200 import binding as B
+    m = W.JAMBA_LIKE
+    ctx = B.Context(m, 16 * W.GiB, 0.3, 16384, max_requests=1024, max_pages=256, device=dev)
+    s0 = ctx.stats()
+    n_req = s0["cap_ssm"] // m.n_ssm_layers
+    per = min(256, s0["cap_kv"] // n_req)
+    st = np.zeros(1024, np.uint32)
+    ctx.step_host(W.make_ops(W.OP_ADMIT, np.arange(n_req), per * 16), n_req, st)
+    assert (st[:n_req] == 0).all()
+    fin = np.arange(0, n_req, 2)
+    ctx.step_host(W.make_ops(W.OP_FINISH, fin, 0), len(fin), st)
+    ops = W.make_ops(W.OP_ADMIT, 512 + np.arange(n_req), 16)
+    d_ops = torch.from_numpy(ops.view(np.uint8).reshape(-1)).to(dev)
+    d_st = torch.zeros(n_req, dtype=torch.int32, device=dev)
+    torch.cuda.synchronize(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    ctx.step(d_ops, n_req, d_st)
+    e1.record()
+    torch.cuda.synchronize(dev)
+    s = ctx.stats()
+    ms = e0.elapsed_time(e1)
+    ctx.close()
+    moved = 2 * s["relocated_bytes"]
+    peak, _ = _peaks()
+    copy_s = s["relocation_ns_last"] * 1e-9
+    return {"relocated_blocks": s["relocated_blocks"], "relocated_bytes": s["relocated_bytes"],
+            "rebalances": s["n_rebalance"], "step_ms": ms,
+            "gbs_whole_step": moved / (ms * 1e-3) / 1e9,
+            "copy_kernel_ms_device_clock": copy_s * 1e3,
+            "gbs_copy_kernel": moved / copy_s / 1e9 if copy_s > 0 else None,
+            "frac_of_peak_copy_kernel": moved / copy_s / 1e9 / peak if copy_s > 0 else None,
+            "note": "one avmp_step whose CapacityError migrates 16384 KV pages; whole step = plan kernel + copy "
+                    "(CUDA events); copy kernel alone by the device clock stamped inside it (first warp in, last out)"}
+
+
+def allocator_scaling(dev, batches=(32, 256, 1024, 4096), warm=120, timed=60) -> list:
+    """avmp_step alone on closed-loop traces of growing step batch (small units so that
+    thousands of requests fit): the path is latency-bound, so ops/s grows with the batch."""
+    import torch
+    from paper_2605_22416_b200 import binding as B
+    out = []
+    for n in batches:
+        w = W.Workload(f"alloc_micro_{n}", W.SMALL_UNIT_MODEL, 1 * W.GiB, 0.5, 128, n, n, 24, "queue", 400 * n)
+        ctx = B.Context.from_workload(w, device=dev)
+        drv = W.ClosedLoopDriver(w)
+        trace = []
+        while not drv.done and drv.step < warm + timed:
+            ops = drv.next_batch()
+            st = np.zeros(len(ops), np.uint32)
+            ctx.step_host(np.ascontiguousarray(ops), len(ops), st)
+            drv.feed(st)
+            trace.append(ops)
+        s_a = ctx.stats()
+        ctx.close()
+        ctx = B.Context.from_workload(w, device=dev)
+        d_ops = [torch.from_numpy(np.ascontiguousarray(o).view(np.uint8).reshape(-1)).to(dev) if len(o) else None for o in trace]
+        d_st = torch.zeros(2 * n + 16, dtype=torch.int32, device=dev)
+        sid = torch.cuda.current_stream().cuda_stream
+        for o, d in zip(trace[:warm], d_ops[:warm]):
+            ctx.step(d, len(o), d_st, sid)
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for o, d in zip(trace[warm:], d_ops[warm:]):
+            ctx.step(d, len(o), d_st, sid)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        s_b = ctx.stats()
+        ctx.close()
+        n_ops = sum(len(o) for o in trace[warm:])
+        ms = e0.elapsed_time(e1)
+        out.append({"step_batch": n, "ops_per_step": n_ops / max(len(trace) - warm, 1), "us_per_step": ms * 1e3 / max(len(trace) - warm, 1),
+                    "ops_per_s": n_ops / (ms * 1e-3), "n_oom": s_b["n_oom"], "rebalances": s_b["n_rebalance"],
+                    "replay_matches": all(s_b[k] == s_a[k] for k in ("n_oom", "n_rebalance", "op_counter", "free_kv", "free_ssm"))})
+    return out
+
+
+# ---------------------------------------------------------------------------------------
 # the oracle on the host cores: cpu_baseline leg and the --impl reference arm
 # ---------------------------------------------------------------------------------------
 def run_oracle(args, n_sample_steps: int, budget_s: float = 25.0) -> dict:
@@ -433,6 +519,7 @@ def main():
     ap.add_argument("--workload", default="short_uniform")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-micro", action="store_true", help="skip the migration and allocator micro-benchmarks")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -452,6 +539,11 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     out = run_ours(args, rank, world, local_rank)
     if rank == 0:
+        if not args.no_micro:
+            import torch
+            dev = torch.device("cuda", local_rank)
+            out["migration"]["microbench"] = migration_microbench(dev)
+            out["allocator"]["vs_step_batch"] = allocator_scaling(dev)
         if not args.no_cpu_baseline:
             out["cpu_baseline"] = run_oracle(args, n_sample_steps=12)
         print(json.dumps(out), flush=True)

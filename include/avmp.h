@@ -137,6 +137,8 @@ typedef struct {
     uint64_t pool_bytes_aligned;
     uint64_t error_code;          /* first AVMP_DEV_* error seen, sticky */
     uint64_t error_count;         /* items skipped because of device-side errors */
+    uint64_t relocation_ns_last;  /* device-clock duration of the last relocation copy (first CTA in, last out) */
+    uint64_t relocation_ns_total; /* sum over all relocation copies: the time spent migrating payload */
 } avmp_stats;
 #define AVMP_N_STATS (sizeof(avmp_stats) / sizeof(uint64_t))
 

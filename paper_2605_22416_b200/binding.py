@@ -26,7 +26,7 @@ STAT_FIELDS = (
     "migrated_bytes", "wasted_bytes", "relocated_blocks", "relocated_bytes", "gap_bytes",
     "cap_kv", "cap_ssm", "free_kv", "free_ssm", "fsm_state", "n_invalid",
     "unit_bytes_kv", "unit_bytes_ssm", "vid_space_kv", "vid_space_ssm", "pool_bytes_aligned",
-    "error_code", "error_count",
+    "error_code", "error_count", "relocation_ns_last", "relocation_ns_total",
 )
 
 

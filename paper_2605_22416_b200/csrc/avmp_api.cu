@@ -74,6 +74,9 @@ void fill_stats(const avmp_ctx *c, const DevState &d, avmp_stats *o)
     o->fsm_state = d.fsm; o->n_invalid = d.n_invalid;
     o->pool_bytes_aligned = c->lay.pool_bytes_aligned;
     o->error_code = d.error_code; o->error_count = d.error_count;
+    const uint64_t last = (d.reloc_t1 > d.reloc_t0 && d.reloc_t0 != kNone64) ? d.reloc_t1 - d.reloc_t0 : 0;
+    o->relocation_ns_last = last;
+    o->relocation_ns_total = d.reloc_ns_total + (d.reloc_pending ? last : 0);
 }
 
 }  // namespace

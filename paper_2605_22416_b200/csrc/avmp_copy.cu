@@ -59,6 +59,7 @@ struct Piece {
 // layers (layer-major piece order; layer l's buffers start l * stride bytes further on).
 template <bool SCATTER>
 struct SsmPieces {
+    static constexpr bool kTimed = false;
     uint32_t layer0, n_layers, n, ps, per;
     const uint32_t *reqs;
     uint8_t *buf_state, *buf_conv;
@@ -98,6 +99,7 @@ struct SsmPieces {
 
 // a7: chunks of the units moved by the last migration.
 struct RelocPieces {
+    static constexpr bool kTimed = true;     // the copy stamps the device clock: migration time is a metric
     __device__ unsigned long long total(const Geom &g) const
     {
         const unsigned long long U = g.U[g.st->reloc_pool];
@@ -122,6 +124,7 @@ struct RelocPieces {
 // (K slices, then V slices).
 template <bool SCATTER>
 struct KvPieces {
+    static constexpr bool kTimed = false;
     uint32_t layer0, n_layers, n, subs;
     const uint32_t *reqs, *tok_start;
     uint8_t *buf_k, *buf_v;
@@ -276,6 +279,7 @@ __global__ void __launch_bounds__(kBulkThreads, kBulkCtasPerSm) stream_bulk_kern
     const unsigned long long first = (unsigned long long)warp * gridDim.x + blockIdx.x;
     const unsigned long long stride = (unsigned long long)gridDim.x * kBulkWarps;
     if (first >= total) return;
+    if (F::kTimed && lane == 0) atomicMin(&g.st->reloc_t0, global_ns());
     const unsigned long long mine = (total - first + stride - 1) / stride;       // pieces of this warp
     const uint32_t n_batches = (uint32_t)((mine + kBatch - 1) / kBatch);
 
@@ -310,6 +314,7 @@ __global__ void __launch_bounds__(kBulkThreads, kBulkCtasPerSm) stream_bulk_kern
         while (!ring.failed && ring.n_stored < ring.n_loaded) ring.retire_one();
         if (ring.failed) record_error(g.st, AVMP_DEV_TIMEOUT);
         bulk_wait_all();
+        if (F::kTimed) atomicMax(&g.st->reloc_t1, global_ns());
     }
 }
 
@@ -320,7 +325,9 @@ __global__ void __launch_bounds__(kGenThreads) stream_generic_kernel(const Geom 
     pdl_prologue();
     const unsigned long long total = f.total(g);
     const unsigned long long nw = (unsigned long long)gridDim.x * (kGenThreads / 32);
-    for (unsigned long long it = (unsigned long long)(threadIdx.x >> 5) * gridDim.x + blockIdx.x; it < total; it += nw) {
+    const unsigned long long it0 = (unsigned long long)(threadIdx.x >> 5) * gridDim.x + blockIdx.x;
+    if (F::kTimed && lane == 0 && it0 < total) atomicMin(&g.st->reloc_t0, global_ns());
+    for (unsigned long long it = it0; it < total; it += nw) {
         Piece p{nullptr, nullptr, 0};
         if (lane == 0) p = f.get(g, it);
         p.src = (const uint8_t *)__shfl_sync(0xFFFFFFFFu, (unsigned long long)p.src, 0);
@@ -334,6 +341,7 @@ __global__ void __launch_bounds__(kGenThreads) stream_generic_kernel(const Geom 
             for (uint32_t i = lane; i < p.bytes; i += 32u) p.dst[i] = p.src[i];
         }
     }
+    if (F::kTimed && lane == 0 && it0 < total) { __threadfence(); atomicMax(&g.st->reloc_t1, global_ns()); }
 }
 
 template <class F>

@@ -20,12 +20,13 @@ struct DevState {
     unsigned long long op_counter, last_rebalance_op, n_oom, n_capacity_error, n_rebalance;
     unsigned long long migrated_bytes, wasted_bytes, relocated_blocks, relocated_bytes, gap_bytes;
     unsigned long long n_invalid, error_code, error_count;
+    unsigned long long reloc_t0, reloc_t1, reloc_ns_total;   // device clock around relocation copies
     uint32_t cap[2], n_free[2], n_vfree[2], fsm;
     uint32_t resume_idx;     // ops of the batch in flight already applied (multi-round steps)
     uint32_t n_reloc;        // relocation list of the last round
     uint32_t reloc_pool;
     uint32_t g_total_items;  // work items of the gather / scatter being planned
-    uint32_t pad;
+    uint32_t reloc_pending;  // reloc_t0 / reloc_t1 hold a copy not yet added to reloc_ns_total
 };
 
 // Immutable geometry + table pointers, passed to kernels by value.
@@ -47,6 +48,13 @@ __device__ __forceinline__ uint8_t *unit_ptr(const Geom &g, uint32_t pool, uint3
 {
     return pool == AVMP_POOL_KV ? g.arena + (unsigned long long)slot * g.U[0]
                                 : g.arena + (g.P_al - ((unsigned long long)slot + 1ull) * g.U[1]);
+}
+
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
 }
 
 __device__ __forceinline__ void record_error(DevState *st, unsigned long long code)

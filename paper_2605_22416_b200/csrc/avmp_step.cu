@@ -200,6 +200,10 @@ step_kernel(const Geom g, const avmp_op *__restrict__ ops, const uint32_t n_ops,
         sc.gap = ds->gap_bytes; sc.n_invalid = ds->n_invalid; sc.counter_base = ds->op_counter;
         for (int p = 0; p < 2; ++p) { sc.cap[p] = ds->cap[p]; sc.nfree[p] = ds->n_free[p]; sc.nvfree[p] = ds->n_vfree[p]; }
         sc.fsm = ds->fsm;
+        if (ds->reloc_pending) {            // fold the last relocation copy's duration into the total
+            if (ds->reloc_t1 > ds->reloc_t0) ds->reloc_ns_total += ds->reloc_t1 - ds->reloc_t0;
+            ds->reloc_pending = 0;
+        }
         sc.migs_done = 0; sc.abort = 0; sc.abort_idx = 0; sc.n_reloc = 0; sc.reloc_pool = 0;
         sc.mig = 0;
         sh.excl_k[0] = first_round ? 0u : ds->resume_idx;    // borrow a slot to broadcast the start
@@ -426,6 +430,7 @@ step_kernel(const Geom g, const avmp_op *__restrict__ ops, const uint32_t n_ops,
         ds->resume_idx = done_upto;
         ds->n_reloc = sc.n_reloc;
         ds->reloc_pool = sc.reloc_pool;
+        if (sc.n_reloc) { ds->reloc_t0 = kNone64; ds->reloc_t1 = 0; ds->reloc_pending = 1; }
     }
 }
 

@@ -168,6 +168,7 @@ PR1_MODEL = ModelShape(4, 12, 16, 8, 128, 2, 2048 * 16, 2048 * 3, 4)
 JAMBA_LIKE = ModelShape(4, 28, 16, 8, 128, 2, 8192 * 16, 8192 * 3, 4)
 SCALE_MODEL = ModelShape(9, 63, 16, 8, 128, 2, 16384 * 16, 16384 * 3, 4)
 TINY_MODEL = ModelShape(1, 1, 16, 1, 1, 2, 20, 4, 4)  # 64-byte pages, 96-byte blocks
+SMALL_UNIT_MODEL = ModelShape(1, 2, 16, 1, 64, 2, 256, 64, 4)  # 4 KiB pages, 1280-byte blocks: many units per GiB
 
 MiB = 1 << 20
 GiB = 1 << 30
@@ -244,6 +245,9 @@ def make_requests(w: Workload, n: Optional[int] = None) -> RequestList:
     elif w.name == "tiny":
         p = rand_int(s, 1, n, 1, 70)
         o = rand_int(s, 2, n, 1, 20)
+    elif w.name.startswith("alloc_micro"):
+        p = rand_int(s, 1, n, 16, 256)
+        o = rand_int(s, 2, n, 16, 128)
     else:
         raise ValueError(f"no queue recipe for {w.name}")
     return RequestList(p.astype(np.int64), o.astype(np.int64))
