@@ -32,9 +32,10 @@ from paper_2605_22416_b200 import workloads as W  # noqa: E402
 
 METRIC = "paged gather+migration GB/s over whole engine steps (allocator ops/s reported beside it)"
 WARM_STEPS = 600          # closed-loop steps before the measured window (steady state)
-# DRAM bytes (read + write) per launch of the dominant kernel divided by its algorithmic bytes,
-# from the ncu capture summarised in profiles/ssm_gather_short_uniform.md; None until measured.
-NCU_TRAFFIC_RATIO = None
+# DRAM bytes (read + write) per launch of the dominant kernel divided by its algorithmic bytes, from the
+# ncu capture summarised in profiles/ssm_gather_fused_jamba_like.md (a smaller case of the same kernel:
+# 1.04 GB per launch instead of 6.8 GB; traffic grows in proportion to the blocks gathered).
+NCU_TRAFFIC_RATIO = 0.956
 
 
 def _peaks():

@@ -74,6 +74,8 @@ def main():
         n_req = 150 if args.case != "kv_gather" else 48
         tokens = 64 if args.case != "kv_gather" else 2048
         ctx = B.Context(m, pool, split, 128, max_requests=256, max_pages=256)
+        s0 = ctx.stats()
+        n_req = min(n_req, s0["cap_ssm"] // m.n_ssm_layers, s0["cap_kv"] // (tokens // 16))
         ops = W.make_ops(W.OP_ADMIT, np.arange(n_req), tokens)
         st = np.zeros(n_req, np.uint32)
         ctx.step_host(ops, n_req, st)
