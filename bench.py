@@ -101,6 +101,12 @@ def step_bytes(model: W.ModelShape, n_running: int, total_tokens: int, relocated
     return {"kv": kv, "ssm": ssm, "reloc": 2 * relocated_bytes}
 
 
+def config_dict(w: W.Workload) -> dict:
+    return {"workload": w.name, "model": "jamba-like 4 attn + 28 mamba layers", "pool_gib": w.pool_bytes / W.GiB,
+            "split": w.split, "migration_batch_size": w.migration_batch_size, "step_batch": w.concurrency,
+            "warm_steps": WARM_STEPS}
+
+
 def reduce_over_ranks(local_ms: float, local_sums: np.ndarray, world: int):
     """max of the time, sum of the additive quantities, over all ranks (identity at world 1)."""
     if world == 1:
@@ -318,9 +324,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
         "n_gpus": world, "steps": K, "warmup": args.warmup, "ms_per_step": total_ms_g / K,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u32",
         "data": "synthetic", "impl": "ours",
-        "config": {"workload": w.name, "model": "jamba-like 4 attn + 28 mamba layers", "pool_gib": w.pool_bytes / W.GiB,
-                   "split": w.split, "migration_batch_size": w.migration_batch_size, "step_batch": w.concurrency,
-                   "warm_steps": WARM_STEPS, "running_mean": float(np.mean([len(r["run"]) for r in timed])),
+        "config": {**config_dict(w), "running_mean": float(np.mean([len(r["run"]) for r in timed])),
                    "tokens_mean": float(np.mean([int(r["lens"].sum()) for r in timed])),
                    "l2": "inputs larger than L2 (each step moves GBs across a 4 GiB arena; per-layer outputs are distinct buffers)",
                    "multi_gpu": "replicas only: one independent context per GPU, no collective"},
@@ -504,7 +508,7 @@ def run_reference(args) -> dict:
     return {"metric": METRIC, "value": base["value"], "unit": "GB/s", "n_gpus": args.gpus, "steps": base["steps"],
             "warmup": args.warmup, "ms_per_step": base["ms_per_step"], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "u32", "data": "synthetic", "impl": "reference",
-            "config": {"workload": w.name, "note": "the CPU oracle as it stands, single thread, bounded sample"},
+            "config": {**config_dict(w), "note": "the CPU oracle as it stands, single thread, bounded sample of the same steps"},
             "cpu_baseline": {k: base[k] for k in ("value", "unit", "cores", "kind", "sample")},
             "allocator": {"ops_per_s": base["allocator_ops_per_s"]},
             "e2e": {"value": base["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
