@@ -130,12 +130,43 @@ def test_many_migrations_inside_one_batch(env):
     assert g.stats()["n_rebalance"] > 15 and g.stats()["relocated_blocks"] > 10
 
 
+def _check_fused_gathers(g, h, d, w, kl, sl):
+    """The multi-layer entry points (the launch configuration the benchmark times) on a range of
+    layers around the written ones: the written layer against the payload function, its
+    neighbours against the single-layer entry point."""
+    run = d.running_slots.astype(np.uint32)
+    if len(run) == 0:
+        return
+    m = w.model
+    lens = d.len[run]
+    tot = int(lens.sum())
+    k0 = max(0, min(kl - 1, m.n_attn_layers - 3))
+    nk = min(3, m.n_attn_layers - k0)
+    gk, gv, gcu = g.gather_kv_layers(k0, nk, run, tot)
+    ek, ev_, ecu = h.expected_kv(kl, d.uid[run], lens)
+    assert np.array_equal(gcu, ecu)
+    assert np.array_equal(gk[kl - k0][:tot], ek) and np.array_equal(gv[kl - k0][:tot], ev_)
+    for l in range(nk):
+        if k0 + l != kl:
+            sk, sv, scu, bad = g.gather_kv(k0 + l, run, tot)
+            assert bad == 0 and np.array_equal(gk[l][:tot], sk) and np.array_equal(gv[l][:tot], sv)
+    s0 = max(0, min(sl - 1, m.n_ssm_layers - 3))
+    ns = min(3, m.n_ssm_layers - s0)
+    gs, gc = g.gather_ssm_layers(s0, ns, run)
+    es, ec = h.expected_ssm(sl, d.uid[run], d.slot_epoch[run])
+    assert np.array_equal(gs[sl - s0], es) and np.array_equal(gc[sl - s0], ec)
+    for l in range(ns):
+        if s0 + l != sl:
+            ss, sc_, bad = g.gather_ssm(s0 + l, run)
+            assert bad == 0 and np.array_equal(gs[l], ss) and np.array_equal(gc[l], sc_)
+
+
 def _closed_loop_parity(env, w, steps, *, with_store, kv_layers, ssm_layers, table_every, gather_every,
                         max_migration_checks=10**9):
     g, o = _pair(env, w, with_store=with_store)
     engines = [g, o] if with_store else [g]
     h = PayloadHarness(w, engines, kv_layers=kv_layers, ssm_layers=ssm_layers)
-    seen = dict(reb=0, tokens=0, mig_checks=0)
+    seen = dict(reb=0, tokens=0, mig_checks=0, fused=0)
 
     def step(ops):
         so = o.step(ops)
@@ -160,6 +191,9 @@ def _closed_loop_parity(env, w, steps, *, with_store, kv_layers, ssm_layers, tab
             kl = kv_layers[d.step % len(kv_layers)]
             sl = ssm_layers[d.step % len(ssm_layers)]
             seen["tokens"] += h.check_gathers(d, kl, sl)
+            if seen["fused"] < 3 and len(d.running_slots) > 1:      # a few times per run: it moves GBs to the host
+                seen["fused"] += 1
+                _check_fused_gathers(g, h, d, w, kl, sl)
             if with_store:
                 # the two implementations against each other, including translate of live handles
                 run = d.running_slots.astype(np.uint32)
