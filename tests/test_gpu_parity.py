@@ -80,6 +80,46 @@ def test_random_op_strings_tiny(env, seed, batch):
     check_invariants(s, g.tables(), page_tokens=16, n_ssm_layers=1, max_pages=8)
 
 
+@pytest.mark.parametrize("split", [0.0, 1.0])
+def test_one_pool_starts_empty(env, split):
+    """Degenerate split: one store starts with zero capacity."""
+    w = W.config("tiny", pool_bytes=2048, split=split, migration_batch_size=4)
+    g, o = _pair(env, w, max_requests=6, max_pages=8)
+    ops = W.random_op_string(7, 1200, 6, 50)
+    for i in range(0, len(ops), 40):
+        b = ops[i:i + 40]
+        assert np.array_equal(g.step(b), o.step(b)), i
+        env["same"](g, o, w, f"batch at {i}")
+    assert g.stats()["n_rebalance"] >= 5
+
+
+def test_longest_chain_and_full_pools(env):
+    """Maximum sizes: a chain that fills max_pages exactly, one page more (TOO_LONG), a pool
+    filled to its last unit, and the largest batch the host entry point accepts."""
+    w = W.config("pr1", pool_bytes=64 * W.MiB, migration_enabled=False)
+    g, o = _pair(env, w)
+    cap_kv = o.stats()["cap_kv"]
+    assert cap_kv == 128
+    ops = np.concatenate([
+        W.make_ops(W.OP_ADMIT, [0], 40 * 16),            # exactly max_pages
+        W.make_ops(W.OP_EXTEND, [0], 1),                 # one more page: TOO_LONG
+        W.make_ops(W.OP_ADMIT, [1], 40 * 16),
+        W.make_ops(W.OP_ADMIT, [2], 40 * 16),
+        W.make_ops(W.OP_ADMIT, [3], 8 * 16),             # the pool's last 8 pages
+        W.make_ops(W.OP_ADMIT, [4], 1),                  # nothing left: OOM
+        W.make_ops(W.OP_FINISH, [1], 0),
+        W.make_ops(W.OP_ADMIT, [4], 40 * 16 + 1),        # 41 pages: TOO_LONG before any capacity check
+        W.make_ops(W.OP_ADMIT, [4], 40 * 16),
+    ])
+    sg, so = g.step(ops), o.step(ops)
+    assert np.array_equal(sg, so) and so.tolist() == [0, 3, 0, 0, 0, 1, 0, 3, 0]
+    env["same"](g, o, w, "full pools")
+    assert g.stats()["free_kv"] == 0
+    big = W.random_op_string(3, 65536, 32, 200)
+    assert np.array_equal(g.step_host(big), o.step(big))
+    env["same"](g, o, w, "65536-op batch")
+
+
 def test_many_migrations_inside_one_batch(env):
     """min_interval 1: a single batch holds many migrations in both directions, so the step
     runs as several plan/copy rounds; payload must follow every relocation."""
@@ -299,6 +339,36 @@ def test_scale_config(env, split, enabled):
     s, seen, d = _closed_loop_parity(env, w, 120 if enabled else 60, with_store=False, kv_layers=[4],
                                      ssm_layers=[31], table_every=40, gather_every=59, max_migration_checks=6)
     assert seen["tokens"] > 0 and s["op_counter"] > 40_000
+
+
+def test_sensitivity_sweep_cells_match_the_oracle(env):
+    """The sweep of Section 4.5 (migration_batch_size, thresholds, static partition): every cell's
+    summary from the GPU run equals the oracle's on the same closed loop, B = 1 behaves like the
+    static partition, and changing threshold_low changes nothing."""
+    from paper_2605_22416_b200 import sweep
+    base = W.config("pr1", pool_bytes=96 * W.MiB, min_rebalance_interval_ops=100)
+    rows_g, rows_o = [], []
+    for w in sweep.cells(base, "all"):
+        rows_g.append(sweep.gpu_cell(w, 400))
+        o = env["Oracle"].from_workload(w)
+        r = sweep.run_cell(w, o.step, o.stats, 400)
+        rows_o.append(r)
+    for a, b in zip(rows_g, rows_o):
+        for k in b:
+            if k != "relocation_ms":
+                assert a[k] == b[k], (k, a, b)
+    static, b1 = rows_o[0], rows_o[1]
+    assert not static["dynamic"] and b1["B"] == 1
+    # one 152 KiB SSM block cannot make a 256 KiB KV page: B = 1 never migrates here and equals the
+    # static partition event for event (the paper's B = 1 row equals its static total too)
+    assert all(b1[k] == static[k] for k in ("n_oom", "rebalances", "completed", "ops", "cap_kv", "cap_ssm"))
+    assert any(r["rebalances"] > 0 and r["relocated_mib"] > 0 for r in rows_o)
+    th = [r for r in rows_o if r["dynamic"] and r["B"] == base.migration_batch_size]
+    ref = {k: v for k, v in th[0].items() if k not in ("th_low",)}
+    same_high = [r for r in th if r["th_high"] == th[0]["th_high"]]
+    assert len(same_high) >= 3
+    for r in same_high:
+        assert {k: v for k, v in r.items() if k != "th_low"} == ref   # stage-2 null result
 
 
 def test_edge_cases(env):

@@ -233,6 +233,25 @@ def test_naive_model_on_tiny_inputs(seed, B):
     assert o.stats()["n_rebalance"] > 0 or B == 1
 
 
+@pytest.mark.parametrize("split", [0.0, 1.0])
+def test_one_pool_starts_empty(split):
+    """Degenerate split: one store has no capacity at all until the first CapacityError moves
+    some over.  Same brute-force comparison as above."""
+    w = W.config("tiny", pool_bytes=2048, split=split, migration_batch_size=4)
+    o = Oracle.from_workload(w, max_requests=6, max_pages=8)
+    nv = M.NaiveAllocator(w.model, w.pool_bytes, w.split, 4, 6, 8, min_interval=4)
+    s0 = o.stats()
+    assert (s0["cap_kv"] == 0) != (s0["cap_ssm"] == 0)
+    ops = W.random_op_string(7, 400, 6, 50)
+    for i in range(len(ops)):
+        st = int(o.step(ops[i:i + 1])[0])
+        assert st == nv.op(int(ops["kind"][i]), int(ops["flags"][i]), int(ops["req"][i]), int(ops["tokens"][i]))
+        _inv(o, w.with_(max_pages=8))
+    s = o.stats()
+    assert s["n_rebalance"] >= 5 and s["relocated_blocks"] > 0 and s["cap_kv"] > 0 and s["cap_ssm"] > 0
+    assert (s["cap_kv"], s["cap_ssm"]) == tuple(nv.cap) and s["relocated_blocks"] == nv.relocated
+
+
 @pytest.mark.parametrize("name,steps", [("pr1", 700), ("short_uniform", 250), ("mixed_long", 400),
                                         ("agentic_burst", 500), ("scale", 60)])
 def test_static_equivalence(name, steps):
