@@ -412,6 +412,42 @@ def migration_microbench(dev) -> dict:
                     "(CUDA events); copy kernel alone by the device clock stamped inside it (first warp in, last out)"}
 
 
+def device_closed_loop(dev, workload: str, steps: int = 3000) -> dict:
+    """The whole serving loop on the device (batch built, allocator stepped and statuses folded back by
+    kernels, no host round trip), dynamic rebalancing against the static partition on the same trace:
+    requests completed in the same number of engine steps, and the device time those steps took."""
+    import torch
+    from paper_2605_22416_b200 import binding as B
+    out = {"workload": workload, "steps": steps}
+    for label, enabled in (("dynamic", True), ("static", False)):
+        w = W.config(workload, migration_enabled=enabled)
+        reqs = W.make_requests(w, min(w.n_requests, 200_000))
+        ctx = B.Context.from_workload(w, device=dev)
+        dd = B.DeviceDriver(ctx, reqs.prompt, reqs.output, w.concurrency)
+        sid = torch.cuda.current_stream().cuda_stream
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            dd.step(sid)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        ms = e0.elapsed_time(e1)
+        ds, st = dd.stats(), ctx.stats()
+        out[label] = {"completed": ds["completed"], "n_oom": st["n_oom"], "rebalances": st["n_rebalance"],
+                      "ops": st["op_counter"], "device_ms": ms, "us_per_step": ms * 1e3 / steps,
+                      "ops_per_s": st["op_counter"] / (ms * 1e-3),
+                      "completed_per_s_allocator_only": ds["completed"] / (ms * 1e-3),
+                      "relocation_ms": st["relocation_ns_total"] / 1e6}
+        dd.close()
+        ctx.close()
+    out["completed_ratio_dynamic_over_static"] = out["dynamic"]["completed"] / max(out["static"]["completed"], 1)
+    out["note"] = ("allocator-only loop: no model kernels and no gathers run between steps, so the per-second figures "
+                   "are a ceiling on scheduling rate, not serving goodput; the ratio of completed requests is the "
+                   "event-deterministic part")
+    return out
+
+
 def allocator_scaling(dev, batches=(32, 256, 1024, 4096), warm=120, timed=60) -> list:
     """avmp_step alone on closed-loop traces of growing step batch (small units so that
     thousands of requests fit): the path is latency-bound, so ops/s grows with the batch."""
@@ -566,6 +602,7 @@ def main():
             dev = torch.device("cuda", local_rank)
             out["migration"]["microbench"] = migration_microbench(dev)
             out["allocator"]["vs_step_batch"] = allocator_scaling(dev)
+            out["closed_loop_device"] = device_closed_loop(dev, args.workload)
         if not args.no_cpu_baseline:
             out["cpu_baseline"] = run_oracle(args, n_sample_steps=12)
         print(json.dumps(out), flush=True)

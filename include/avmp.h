@@ -198,6 +198,12 @@ AVMP_API int avmp_destroy(avmp_ctx *ctx);
  * Stream-ordered, no host synchronisation.  n_ops == 0 is a no-op. */
 AVMP_API int avmp_step(avmp_ctx *ctx, const avmp_op *d_ops, uint32_t n_ops, uint32_t *d_status, void *stream);
 
+/* Same step, with the batch length read from device memory when the kernel runs (*d_n_ops, clamped
+ * to max_ops): for batches that another kernel builds, so that a serving loop needs no host round
+ * trip per step.  max_ops bounds the work the host queues (the number of migration rounds). */
+AVMP_API int avmp_step_indirect(avmp_ctx *ctx, const avmp_op *d_ops, const uint32_t *d_n_ops, uint32_t max_ops,
+                                uint32_t *d_status, void *stream);
+
 /* Same step with HOST arrays: copies the ops in, runs the step, copies the statuses out
  * and waits for them.  n_ops is limited to 65536 per call. */
 AVMP_API int avmp_step_host(avmp_ctx *ctx, const avmp_op *h_ops, uint32_t n_ops, uint32_t *h_status, void *stream);
@@ -273,6 +279,36 @@ AVMP_API int avmp_clear_error(avmp_ctx *ctx, void *stream);
 /* Tables <-> host (parity checks, snapshot / restore).  Both synchronise the stream. */
 AVMP_API int avmp_export_tables(avmp_ctx *ctx, avmp_tables *h_out, void *stream);
 AVMP_API int avmp_import_tables(avmp_ctx *ctx, const avmp_tables *h_in, void *stream);
+
+/* ---- on-device closed loop (the paper's harness drives its traces from the host, Section 4.1) ----
+ * A device-resident scheduler for queue-type traces: every avmp_driver_step builds the next batch
+ * on the GPU (FINISH for requests whose decode is complete, EXTEND by one token for the other
+ * running requests, ADMITs from the queue head into the lowest free slots within the concurrency
+ * and a slow-start window), runs it through the allocator (avmp_step_indirect) and folds the
+ * statuses back into the request slots -- three stream-ordered launches and no host round trip, so
+ * a serving loop can be queued (or graph-captured) many steps ahead.  d_prompt / d_output are
+ * device arrays of n_requests token counts; the driver's slots are the context's request slots.
+ * The workspace (avmp_driver_workspace_bytes(max_requests), 256-byte aligned) is the caller's. */
+typedef struct avmp_driver avmp_driver;
+typedef struct {
+    uint64_t steps, completed, dropped, preempted, n_oom_admit, n_oom_extend;
+    uint64_t queue_next;      /* requests taken from the arrays so far */
+    uint64_t requeued;        /* entries waiting at the queue head (failed admits, pre-empted requests) */
+    uint64_t window;          /* current admission window */
+    uint64_t last_batch_ops;
+    uint64_t overflow;        /* 1 if the re-queue buffer ever overflowed (entries were lost) */
+} avmp_driver_stats;
+AVMP_API size_t avmp_driver_workspace_bytes(uint32_t max_requests);
+AVMP_API int avmp_driver_create(avmp_driver **out, avmp_ctx *ctx, const uint32_t *d_prompt, const uint32_t *d_output,
+                                uint32_t n_requests, uint32_t concurrency, void *d_workspace, size_t workspace_bytes,
+                                void *stream);
+AVMP_API int avmp_driver_destroy(avmp_driver *drv);
+AVMP_API int avmp_driver_step(avmp_driver *drv, void *stream);
+/* Both synchronise the stream.  Export copies the per-slot arrays (state 0 free / 1 running, request
+ * index, tokens held, decode tokens left), max_requests entries each. */
+AVMP_API int avmp_driver_get_stats(avmp_driver *drv, avmp_driver_stats *h_out, void *stream);
+AVMP_API int avmp_driver_export(avmp_driver *drv, uint32_t *h_state, uint32_t *h_uid, uint32_t *h_len,
+                                uint32_t *h_remaining, void *stream);
 
 /* How many kernels this context has launched so far (host counter). */
 AVMP_API uint64_t avmp_launch_count(const avmp_ctx *ctx);

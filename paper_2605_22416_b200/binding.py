@@ -53,6 +53,14 @@ class avmp_stats(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in STAT_FIELDS]
 
 
+DRIVER_STAT_FIELDS = ("steps", "completed", "dropped", "preempted", "n_oom_admit", "n_oom_extend", "queue_next",
+                      "requeued", "window", "last_batch_ops", "overflow")
+
+
+class avmp_driver_stats(C.Structure):
+    _fields_ = [(n, C.c_uint64) for n in DRIVER_STAT_FIELDS]
+
+
 _u32p = C.POINTER(C.c_uint32)
 
 
@@ -76,6 +84,13 @@ def _load():
         "avmp_destroy": (C.c_int, [vp]),
         "avmp_step": (C.c_int, [vp, vp, C.c_uint32, vp, vp]),
         "avmp_step_host": (C.c_int, [vp, vp, C.c_uint32, vp, vp]),
+        "avmp_step_indirect": (C.c_int, [vp, vp, vp, C.c_uint32, vp, vp]),
+        "avmp_driver_workspace_bytes": (C.c_size_t, [C.c_uint32]),
+        "avmp_driver_create": (C.c_int, [C.POINTER(vp), vp, vp, vp, C.c_uint32, C.c_uint32, vp, C.c_size_t, vp]),
+        "avmp_driver_destroy": (C.c_int, [vp]),
+        "avmp_driver_step": (C.c_int, [vp, vp]),
+        "avmp_driver_get_stats": (C.c_int, [vp, C.POINTER(avmp_driver_stats), vp]),
+        "avmp_driver_export": (C.c_int, [vp, vp, vp, vp, vp, vp]),
         "avmp_translate": (C.c_int, [vp, vp, C.c_uint32, vp, vp, vp, vp]),
         "avmp_gather_kv": (C.c_int, [vp, C.c_uint32, vp, C.c_uint32, vp, vp, C.c_uint64, vp, vp]),
         "avmp_gather_kv_static": (C.c_int, [vp, C.c_uint32, vp, C.c_uint32, vp, vp, C.c_uint64, vp, vp]),
@@ -168,6 +183,43 @@ def avmp_step(ctx, d_ops, n_ops, d_status, stream=None):
 
 def avmp_step_host(ctx, h_ops, n_ops, h_status, stream=None):
     _check(lib.avmp_step_host(ctx, _ptr(h_ops), n_ops, _ptr(h_status), _stream(stream)), "avmp_step_host")
+
+
+def avmp_step_indirect(ctx, d_ops, d_n_ops, max_ops, d_status, stream=None):
+    _check(lib.avmp_step_indirect(ctx, _ptr(d_ops), _ptr(d_n_ops), max_ops, _ptr(d_status), _stream(stream)),
+           "avmp_step_indirect")
+
+
+def avmp_driver_workspace_bytes(max_requests: int) -> int:
+    return lib.avmp_driver_workspace_bytes(max_requests)
+
+
+def avmp_driver_create(ctx, d_prompt, d_output, n_requests, concurrency, d_workspace, workspace_bytes, stream=None) -> int:
+    h = C.c_void_p()
+    _check(lib.avmp_driver_create(C.byref(h), ctx, _ptr(d_prompt), _ptr(d_output), n_requests, concurrency,
+                                  _ptr(d_workspace), workspace_bytes, _stream(stream)), "avmp_driver_create")
+    return h.value
+
+
+def avmp_driver_destroy(drv):
+    _check(lib.avmp_driver_destroy(drv), "avmp_driver_destroy")
+
+
+def avmp_driver_step(drv, stream=None):
+    _check(lib.avmp_driver_step(drv, _stream(stream)), "avmp_driver_step")
+
+
+def avmp_driver_get_stats(drv, stream=None) -> dict:
+    s = avmp_driver_stats()
+    _check(lib.avmp_driver_get_stats(drv, C.byref(s), _stream(stream)), "avmp_driver_get_stats")
+    return {k: int(getattr(s, k)) for k in DRIVER_STAT_FIELDS}
+
+
+def avmp_driver_export(drv, max_requests: int, stream=None) -> dict:
+    a = {k: np.zeros(max_requests, np.uint32) for k in ("state", "uid", "len", "remaining")}
+    _check(lib.avmp_driver_export(drv, _ptr(a["state"]), _ptr(a["uid"]), _ptr(a["len"]), _ptr(a["remaining"]),
+                                  _stream(stream)), "avmp_driver_export")
+    return a
 
 
 def avmp_translate(ctx, d_handles, n, d_pool, d_offset, d_arena_offset=None, stream=None):
@@ -381,3 +433,42 @@ class Context:
 
     def launch_count(self) -> int:
         return avmp_launch_count(self.handle)
+
+
+class DeviceDriver:
+    """Owner of an on-device closed loop over a Context: uploads the request lengths, allocates the
+    driver workspace, forwards to the avmp_driver_* entry points."""
+
+    def __init__(self, ctx: Context, prompt: np.ndarray, output: np.ndarray, concurrency: int):
+        self.ctx = ctx
+        dev = ctx.device
+        self.d_prompt = torch.from_numpy(np.ascontiguousarray(prompt, dtype=np.uint32).view(np.int32)).to(dev)
+        self.d_output = torch.from_numpy(np.ascontiguousarray(output, dtype=np.uint32).view(np.int32)).to(dev)
+        ws = avmp_driver_workspace_bytes(ctx.opt.max_requests)
+        if ws == 0:
+            raise AvmpError("avmp_driver_workspace_bytes rejected max_requests")
+        with torch.cuda.device(dev):
+            self.workspace = torch.empty(ws, dtype=torch.uint8, device=dev)
+            self.handle = avmp_driver_create(ctx.handle, self.d_prompt, self.d_output, len(prompt), concurrency,
+                                             self.workspace, ws)
+
+    def step(self, stream=None):
+        avmp_driver_step(self.handle, stream)
+
+    def stats(self, stream=None) -> dict:
+        return avmp_driver_get_stats(self.handle, stream)
+
+    def export(self, stream=None) -> dict:
+        return avmp_driver_export(self.handle, self.ctx.opt.max_requests, stream)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            torch.cuda.synchronize(self.ctx.device)
+            avmp_driver_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -197,18 +197,16 @@ int avmp_destroy(avmp_ctx *c)
     return AVMP_OK;
 }
 
-int avmp_step(avmp_ctx *c, const avmp_op *d_ops, uint32_t n_ops, uint32_t *d_status, void *stream)
+static int step_rounds(avmp_ctx *c, const avmp_op *d_ops, uint32_t n_ops, const uint32_t *d_n_ops,
+                       uint32_t *d_status, void *stream)
 {
-    if (!c) return AVMP_EINVAL;
-    if (n_ops == 0) return AVMP_OK;
-    if (!d_ops || !d_status || ((uintptr_t)d_ops & 3) || ((uintptr_t)d_status & 3)) return AVMP_EINVAL;
     // Section 3.2 throttle: migrations are >= min_interval logical ops apart, so a batch of n ops
     // holds at most (n - 1) / min_interval + 1 of them; one launch performs at most one.
     uint32_t rounds = 1;
     if (c->opt.migration_enabled)
         rounds = (uint32_t)((n_ops - 1) / c->opt.min_rebalance_interval_ops) + 1;
     for (uint32_t r = 0; r < rounds; ++r) {
-        if (launch_step(c->g, d_ops, n_ops, d_status, r == 0, S(stream)) != cudaSuccess) return AVMP_ECUDA;
+        if (launch_step(c->g, d_ops, n_ops, d_n_ops, d_status, r == 0, S(stream)) != cudaSuccess) return AVMP_ECUDA;
         c->launches += 1;
         if (c->opt.migration_enabled) {
             if (launch_relocate(c->g, L(c, stream)) != cudaSuccess) return AVMP_ECUDA;
@@ -216,6 +214,23 @@ int avmp_step(avmp_ctx *c, const avmp_op *d_ops, uint32_t n_ops, uint32_t *d_sta
         }
     }
     return AVMP_OK;
+}
+
+int avmp_step(avmp_ctx *c, const avmp_op *d_ops, uint32_t n_ops, uint32_t *d_status, void *stream)
+{
+    if (!c) return AVMP_EINVAL;
+    if (n_ops == 0) return AVMP_OK;
+    if (!d_ops || !d_status || ((uintptr_t)d_ops & 3) || ((uintptr_t)d_status & 3)) return AVMP_EINVAL;
+    return step_rounds(c, d_ops, n_ops, nullptr, d_status, stream);
+}
+
+int avmp_step_indirect(avmp_ctx *c, const avmp_op *d_ops, const uint32_t *d_n_ops, uint32_t max_ops,
+                       uint32_t *d_status, void *stream)
+{
+    if (!c || max_ops == 0) return AVMP_EINVAL;
+    if (!d_ops || !d_n_ops || !d_status || ((uintptr_t)d_ops & 3) || ((uintptr_t)d_status & 3) || ((uintptr_t)d_n_ops & 3))
+        return AVMP_EINVAL;
+    return step_rounds(c, d_ops, max_ops, d_n_ops, d_status, stream);
 }
 
 int avmp_step_host(avmp_ctx *c, const avmp_op *h_ops, uint32_t n_ops, uint32_t *h_status, void *stream)

@@ -184,14 +184,16 @@ __device__ __forceinline__ void commit_allocs(const Geom &g, Shared &sh, uint32_
 }
 
 __global__ void __launch_bounds__(NT, 1)
-step_kernel(const Geom g, const avmp_op *__restrict__ ops, const uint32_t n_ops,
-            uint32_t *__restrict__ status, const int first_round)
+step_kernel(const Geom g, const avmp_op *__restrict__ ops, const uint32_t n_ops_max,
+            const uint32_t *__restrict__ n_ops_dev, uint32_t *__restrict__ status, const int first_round)
 {
     __shared__ Shared sh;
     Scalars &sc = sh.sc;
     const int tid = threadIdx.x;
     DevState *ds = g.st;
     pdl_prologue();
+    // the batch length is a launch argument, or (device-built batches) a word in device memory
+    const uint32_t n_ops = n_ops_dev ? min(*n_ops_dev, n_ops_max) : n_ops_max;
 
     if (tid == 0) {
         sc.last = ds->last_rebalance_op; sc.n_oom = ds->n_oom; sc.n_ce = ds->n_capacity_error;
@@ -464,10 +466,10 @@ cudaError_t launch_init(const Geom &g, const DevState &init, cudaStream_t s)
     return launch_pdl(init_kernel, dim3(296), dim3(512), 0, s, g, init);
 }
 
-cudaError_t launch_step(const Geom &g, const avmp_op *d_ops, uint32_t n_ops, uint32_t *d_status,
-                        int first_round, cudaStream_t s)
+cudaError_t launch_step(const Geom &g, const avmp_op *d_ops, uint32_t n_ops, const uint32_t *d_n_ops,
+                        uint32_t *d_status, int first_round, cudaStream_t s)
 {
-    return launch_pdl(step_kernel, dim3(1), dim3(NT), 0, s, g, d_ops, n_ops, d_status, first_round);
+    return launch_pdl(step_kernel, dim3(1), dim3(NT), 0, s, g, d_ops, n_ops, d_n_ops, d_status, first_round);
 }
 
 }  // namespace avmp

@@ -371,6 +371,49 @@ def test_sensitivity_sweep_cells_match_the_oracle(env):
         assert {k: v for k, v in r.items() if k != "th_low"} == ref   # stage-2 null result
 
 
+@pytest.mark.parametrize("name,steps,over", [
+    ("pr1", 900, dict(pool_bytes=40 * W.MiB, min_rebalance_interval_ops=100)),       # OOMs, pre-emptions
+    ("pr1", 400, dict(pool_bytes=8 * W.MiB, migration_enabled=False, n_requests=300)),  # unservable drops
+    ("short_uniform", 500, {}),
+    ("mixed_long", 400, dict(migration_batch_size=64)),
+    ("scale", 60, {}),
+])
+def test_device_closed_loop_matches_host_loop(env, name, steps, over):
+    """The on-device scheduler (batch built and statuses folded back by kernels, no host round trip)
+    ends in exactly the state the host-side batch builder reaches against the oracle: allocator
+    tables and counters, request slots, queue position, every scheduler counter."""
+    from paper_2605_22416_b200 import binding as B
+    w = W.config(name, **over)
+    reqs = W.make_requests(w, min(w.n_requests, 40_000))
+    g = env["GpuEngine"](w)
+    dd = B.DeviceDriver(g.ctx, reqs.prompt, reqs.output, w.concurrency)
+    for _ in range(steps):
+        dd.step()
+    o = env["Oracle"].from_workload(w)
+    d = W.ClosedLoopDriver(w, requests=reqs)
+    n = 0
+    while n < steps:
+        ops = d.next_batch()
+        d.feed(o.step(ops))
+        n += 1
+    env["same"](g, o, w, "device loop vs host loop")
+    ds, ex = dd.stats(), dd.export()
+    assert ds["steps"] == steps and ds["overflow"] == 0
+    assert ds["completed"] == d.completed and ds["dropped"] == d.dropped and ds["preempted"] == d.preempted
+    assert ds["n_oom_admit"] == d.n_oom_admit and ds["n_oom_extend"] == d.n_oom_extend
+    assert ds["window"] == d.window
+    assert ds["queue_next"] - ds["requeued"] == d._next - len(d.front)
+    run = d.state == 1
+    assert np.array_equal(ex["state"] == 1, run)
+    assert np.array_equal(ex["uid"][run], d.uid[run].astype(np.uint32))
+    assert np.array_equal(ex["len"][run], d.len[run].astype(np.uint32))
+    assert np.array_equal(ex["remaining"][run], d.remaining[run].astype(np.uint32))
+    assert g.stats()["error_code"] == 0
+    if name == "pr1":
+        assert d.n_oom_admit > 0 and (d.preempted > 0 or d.dropped > 0)
+    dd.close()
+
+
 def test_edge_cases(env):
     w = W.config("tiny")
     g, o = _pair(env, w, with_store=True)
