@@ -35,7 +35,7 @@ WARM_STEPS = 600          # closed-loop steps before the measured window (steady
 # DRAM bytes (read + write) per launch of the dominant kernel divided by its algorithmic bytes, from the
 # ncu capture summarised in profiles/ssm_gather_fused_jamba_like.md (a smaller case of the same kernel:
 # 1.04 GB per launch instead of 6.8 GB; traffic grows in proportion to the blocks gathered).
-NCU_TRAFFIC_RATIO = 0.956
+NCU_TRAFFIC_RATIO = 0.951
 
 
 def _peaks():

@@ -258,9 +258,9 @@ def test_pr1_every_step(env):
     of the running batch (GPU == oracle == payload function) every few steps."""
     w = W.config("pr1")
     s, seen, d = _closed_loop_parity(env, w, None, with_store=True, kv_layers=[0, 3], ssm_layers=[0, 11],
-                                     table_every=1, gather_every=5)
+                                     table_every=1, gather_every=8)
     assert d.completed == 2000 and s["n_rebalance"] > 10 and s["n_oom"] > 100
-    assert seen["tokens"] > 1_000_000
+    assert seen["tokens"] > 500_000
 
 
 def test_pr1_small_pool_relocations(env):
@@ -315,7 +315,7 @@ def test_multi_layer_gathers(env):
     ("mixed_long", 1200, dict(migration_batch_size=4)),
     ("mixed_long", 1200, dict(migration_batch_size=16)),
     ("mixed_long", 1200, dict(migration_batch_size=64)),
-    ("mixed_long", 300, dict(migration_batch_size=16, split=0.1)),   # the mirrored reading of "split"
+    ("mixed_long", 150, dict(migration_batch_size=16, split=0.1)),   # the mirrored reading of "split"
     ("agentic_burst", 1500, {}),
 ])
 def test_full_size_configs(env, name, steps, over):
