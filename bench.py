@@ -434,7 +434,26 @@ def device_closed_loop(dev, workload: str, steps: int = 3000) -> dict:
         torch.cuda.synchronize(dev)
         ms = e0.elapsed_time(e1)
         ds, st = dd.stats(), ctx.stats()
-        out[label] = {"completed": ds["completed"], "n_oom": st["n_oom"], "rebalances": st["n_rebalance"],
+        # the same loop again, 100 steps captured once in a CUDA graph and replayed
+        graph_us = None
+        try:
+            side = torch.cuda.Stream(device=dev)
+            gr = torch.cuda.CUDAGraph()
+            torch.cuda.synchronize(dev)
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(gr, stream=side):
+                    for _ in range(100):
+                        dd.step(side)
+                g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                g0.record(side)
+                for _ in range(10):
+                    gr.replay()
+                g1.record(side)
+            torch.cuda.synchronize(dev)
+            graph_us = g0.elapsed_time(g1) * 1e3 / 1000
+        except Exception as exc:          # graphs are an optimisation of the launch path, not part of the result
+            graph_us = f"capture failed: {type(exc).__name__}"
+        out[label] = {"completed": ds["completed"], "us_per_step_cuda_graph": graph_us, "n_oom": st["n_oom"], "rebalances": st["n_rebalance"],
                       "ops": st["op_counter"], "device_ms": ms, "us_per_step": ms * 1e3 / steps,
                       "ops_per_s": st["op_counter"] / (ms * 1e-3),
                       "completed_per_s_allocator_only": ds["completed"] / (ms * 1e-3),

@@ -414,6 +414,36 @@ def test_device_closed_loop_matches_host_loop(env, name, steps, over):
     dd.close()
 
 
+def test_device_loop_replayed_from_a_cuda_graph(env):
+    """Fifty engine steps of the on-device loop captured once in a CUDA graph and replayed ten
+    times: same final state as five hundred steps of the host loop on the oracle."""
+    torch = env["torch"]
+    from paper_2605_22416_b200 import binding as B
+    w = W.config("pr1", pool_bytes=40 * W.MiB, min_rebalance_interval_ops=100)
+    reqs = W.make_requests(w)
+    g = env["GpuEngine"](w)
+    dd = B.DeviceDriver(g.ctx, reqs.prompt, reqs.output, w.concurrency)
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            for _ in range(50):
+                dd.step(stream)
+    for _ in range(10):
+        graph.replay()
+    torch.cuda.synchronize()
+    o = env["Oracle"].from_workload(w)
+    d = W.ClosedLoopDriver(w, requests=reqs)
+    for _ in range(500):
+        d.feed(o.step(d.next_batch()))
+    env["same"](g, o, w, "graph replay vs host loop")
+    ds = dd.stats()
+    assert ds["steps"] == 500 and ds["completed"] == d.completed and ds["preempted"] == d.preempted
+    assert g.stats()["n_rebalance"] > 0
+    dd.close()
+
+
 def test_edge_cases(env):
     w = W.config("tiny")
     g, o = _pair(env, w, with_store=True)
