@@ -103,8 +103,9 @@ def step_bytes(model: W.ModelShape, n_running: int, total_tokens: int, relocated
 
 def config_dict(w: W.Workload, warm_steps: int = WARM_STEPS) -> dict:
     m = w.model
-    return {"workload": w.name, "model": f"{m.n_attn_layers} attention + {m.n_ssm_layers} mamba layers, "
-                                         f"state {m.ssm_state_elems} + conv {m.ssm_conv_elems} fp32 per layer",
+    return {"workload": w.name, "cache_shape": f"{m.n_attn_layers} attention + {m.n_ssm_layers} mamba layers, "
+                                               f"KV page {m.page_tokens} tok x {m.kv_heads} x {m.head_dim} bf16, "
+                                               f"SSM block {m.ssm_state_elems} + {m.ssm_conv_elems} fp32",
             "pool_gib": w.pool_bytes / W.GiB,
             "split": w.split, "migration_batch_size": w.migration_batch_size, "step_batch": w.concurrency,
             "warm_steps": warm_steps}
