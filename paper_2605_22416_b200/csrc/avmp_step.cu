@@ -23,7 +23,6 @@ namespace avmp {
 
 namespace {
 
-constexpr int NT = kStepThreads;
 constexpr uint32_t INF = 0xFFFFFFFFu;
 constexpr uint32_t ST_PENDING = 0xFFu;
 enum : uint8_t { DIR_NONE = 0, DIR_NOP = 1, DIR_ALLOC = 2, DIR_FREE = 3 };
@@ -38,9 +37,12 @@ struct Scalars {
     unsigned long long mig_waste;
 };
 
-constexpr uint32_t kHash = 2 * NT;     // open-addressing table for same-slot detection
-
+// NT = threads of the planning CTA = ops per window.  Small batches run with a small CTA: the
+// kernel is a chain of some forty block barriers, and a barrier over 8 warps costs a fraction of
+// one over 32.
+template <int NT>
 struct Shared {
+    static constexpr uint32_t kHash = 2 * NT;     // open-addressing table for same-slot detection
     uint32_t excl_k[NT + 1], excl_s[NT + 1];
     uint32_t req[NT], base[NT];
     uint32_t hkey[kHash], hval[kHash];
@@ -61,7 +63,8 @@ __device__ __forceinline__ bool would_migrate(const Geom &g, const Scalars &sc, 
 }
 
 // Section 3.2 handler for a shortage in pool X at logical time `counter`; whole CTA.
-__device__ void capacity_error(const Geom &g, Shared &sh, int X, unsigned long long counter)
+template <int NT>
+__device__ void capacity_error(const Geom &g, Shared<NT> &sh, int X, unsigned long long counter)
 {
     Scalars &sc = sh.sc;
     const int Y = 1 - X;
@@ -152,7 +155,8 @@ __device__ void capacity_error(const Geom &g, Shared &sh, int X, unsigned long l
 }
 
 // Pop units for the ops [lo, hi) of the current alloc scan (none of them fails).
-__device__ __forceinline__ void commit_allocs(const Geom &g, Shared &sh, uint32_t lo, uint32_t hi)
+template <int NT>
+__device__ __forceinline__ void commit_allocs(const Geom &g, Shared<NT> &sh, uint32_t lo, uint32_t hi)
 {
     Scalars &sc = sh.sc;
     const int tid = threadIdx.x;
@@ -183,11 +187,13 @@ __device__ __forceinline__ void commit_allocs(const Geom &g, Shared &sh, uint32_
     __syncthreads();
 }
 
+template <int NT>
 __global__ void __launch_bounds__(NT, 1)
 step_kernel(const Geom g, const avmp_op *__restrict__ ops, const uint32_t n_ops_max,
             const uint32_t *__restrict__ n_ops_dev, uint32_t *__restrict__ status, const int first_round)
 {
-    __shared__ Shared sh;
+    __shared__ Shared<NT> sh;
+    constexpr uint32_t kHash = Shared<NT>::kHash;
     Scalars &sc = sh.sc;
     const int tid = threadIdx.x;
     DevState *ds = g.st;
@@ -246,7 +252,7 @@ step_kernel(const Geom g, const avmp_op *__restrict__ ops, const uint32_t n_ops_
         __syncthreads();
         uint32_t hs = 0;
         if (dir >= DIR_ALLOC) {
-            hs = (req * 2654435761u) >> 21;                      // 11 bits
+            hs = (req * 2654435761u) & (kHash - 1u);
             while (true) {
                 const uint32_t old = atomicCAS(&sh.hkey[hs], INF, req);
                 if (old == INF || old == req) break;
@@ -469,7 +475,11 @@ cudaError_t launch_init(const Geom &g, const DevState &init, cudaStream_t s)
 cudaError_t launch_step(const Geom &g, const avmp_op *d_ops, uint32_t n_ops, const uint32_t *d_n_ops,
                         uint32_t *d_status, int first_round, cudaStream_t s)
 {
-    return launch_pdl(step_kernel, dim3(1), dim3(NT), 0, s, g, d_ops, n_ops, d_n_ops, d_status, first_round);
+    if (n_ops <= 256)
+        return launch_pdl(step_kernel<256>, dim3(1), dim3(256), 0, s, g, d_ops, n_ops, d_n_ops, d_status, first_round);
+    if (n_ops <= 512)
+        return launch_pdl(step_kernel<512>, dim3(1), dim3(512), 0, s, g, d_ops, n_ops, d_n_ops, d_status, first_round);
+    return launch_pdl(step_kernel<1024>, dim3(1), dim3(1024), 0, s, g, d_ops, n_ops, d_n_ops, d_status, first_round);
 }
 
 }  // namespace avmp
