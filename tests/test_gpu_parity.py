@@ -120,6 +120,50 @@ def test_longest_chain_and_full_pools(env):
     env["same"](g, o, w, "65536-op batch")
 
 
+@pytest.mark.parametrize("case", range(10))
+def test_random_shapes_and_policies(env, case):
+    """Random cache shapes (rows that are and are not 16-byte multiples: both copy paths), pool
+    sizes, splits, migration_batch_size, throttle and thresholds; random op batches; payload written
+    and gathered back through both implementations after every batch."""
+    rng = np.random.default_rng(1000 + case)
+    shape = W.ModelShape(int(rng.integers(1, 4)), int(rng.integers(1, 5)), int(rng.choice([4, 16])),
+                         int(rng.integers(1, 3)), int(rng.choice([1, 4, 8, 64])), 2,
+                         int(rng.integers(3, 40)) * (4 if case % 2 else 1), int(rng.integers(1, 9)) * (4 if case % 2 else 1), 4)
+    row = shape.kv_row_bytes
+    u = max(shape.n_attn_layers * 2 * shape.page_tokens * row, (shape.ssm_state_elems + shape.ssm_conv_elems) * 4)
+    pool = int(rng.integers(10, 60)) * u
+    w = W.Workload(f"rand{case}", shape, pool, float(rng.choice([0.0, 0.3, 0.5, 0.7, 1.0])), int(rng.integers(1, 9)),
+                   8, 8, 6, "queue", 0, min_rebalance_interval_ops=int(rng.integers(1, 20)),
+                   threshold_high_ppm=int(rng.choice([100_000, 300_000, 500_000])))
+    g, o = _pair(env, w, with_store=True)
+    for rnd in range(25):
+        ops = W.random_op_string(case * 100 + rnd, int(rng.integers(1, 40)), 8, shape.page_tokens * 3, p_invalid=0.05)
+        assert np.array_equal(g.step(ops), o.step(ops)), (case, rnd)
+        env["same"](g, o, w, f"case {case} round {rnd}")
+        t = o.tables()
+        held = np.flatnonzero(t["req_state"] != 0).astype(np.uint32)
+        live = np.flatnonzero(t["req_state"] == 1).astype(np.uint32)
+        lens = t["req_len"][held]
+        tot = int(lens.sum())
+        for layer in range(shape.n_attn_layers):
+            kb = rng.integers(0, 256, (tot, row), dtype=np.uint8)
+            vb = rng.integers(0, 256, (tot, row), dtype=np.uint8)
+            for e in (g, o):
+                assert e.scatter_kv(layer, held, np.zeros(len(held), np.uint32), kb, vb) == 0
+            gk, gv, gcu, gb = g.gather_kv(layer, held, tot)
+            ok, ov, ocu, ob = o.gather_kv(layer, held, tot)
+            assert gb == ob == 0 and np.array_equal(gcu, ocu)
+            assert np.array_equal(gk, kb) and np.array_equal(gv, vb) and np.array_equal(ok, kb) and np.array_equal(ov, vb)
+        for layer in range(shape.n_ssm_layers):
+            sb = rng.integers(0, 256, (len(live), shape.state_bytes), dtype=np.uint8)
+            cb = rng.integers(0, 256, (len(live), shape.conv_bytes), dtype=np.uint8)
+            for e in (g, o):
+                assert e.scatter_ssm(layer, live, sb, cb) == 0
+            gs, gc, gb = g.gather_ssm(layer, live)
+            assert gb == 0 and np.array_equal(gs, sb) and np.array_equal(gc, cb)
+    assert g.stats()["error_code"] == 0
+
+
 def test_many_migrations_inside_one_batch(env):
     """min_interval 1: a single batch holds many migrations in both directions, so the step
     runs as several plan/copy rounds; payload must follow every relocation."""
