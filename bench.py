@@ -288,9 +288,9 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     # ---- e2e: host buffers in, host results out, every step ----
     ctx = fresh_context(full_warmup=False)
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.uint8).reshape(-1).copy()).pin_memory()
-    h_ops = [np.ascontiguousarray(r["ops"]) for r in timed]
+    h_ops = [pin(r["ops"]) if len(r["ops"]) else torch.zeros(16, dtype=torch.uint8).pin_memory() for r in timed]
     h_run = [pin(r["run"]) for r in timed]
-    h_status = np.zeros(w.concurrency * 2 + 16, np.uint32)
+    h_status = torch.zeros(w.concurrency * 2 + 16, dtype=torch.int32).pin_memory()
     h_cu = torch.zeros(max_run + 1, dtype=torch.int32).pin_memory()
     d_run_buf = torch.zeros(max_run * 4 + 16, dtype=torch.uint8, device=dev)
     h2d = d2h = 0
@@ -361,7 +361,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
                      "traffic": None if NCU_TRAFFIC_RATIO is None else ssm_launch_bytes * NCU_TRAFFIC_RATIO},
         "e2e": {"value": sums[0] / (e2e_ms_g * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms_g / K,
                 "h2d_bytes_per_step": sums[5] / K / world, "d2h_bytes_per_step": sums[6] / K / world,
-                "note": "ops and running list from pinned/pageable host memory, statuses and row offsets back to the host every step; gathered batch buffers stay in HBM for the model's kernels"},
+                "note": "ops and running list from pinned host memory, statuses and row offsets back to the host every step; gathered batch buffers stay in HBM for the model's kernels"},
         "gpu_launches": int(sums[4]),
         "clocks": clocks,
         "replay_matches_closed_loop": all(st_b[k] == stats_a[k] for k in stats_a if not k.startswith("relocation_ns")),

@@ -95,15 +95,24 @@ __device__ void capacity_error(const Geom &g, Shared<NT> &sh, int X, unsigned lo
     unsigned long long tot;
 
     // 1. The donor shrinks at its high end: drop free slots >= newcap, keeping the order.
-    //    In place: a chunk is read in full (the scan's barriers) before it is written, and
-    //    writes never pass the chunk's own start.
+    //    In place, kPer consecutive entries per thread and step: a chunk is read in full (the
+    //    scan's barriers) before it is written, and writes never pass the chunk's own start.
+    constexpr uint32_t kPer = 8;
     uint32_t kept = 0;
-    for (uint32_t b = 0; b < total; b += NT) {
-        const uint32_t i = b + tid;
-        const uint32_t v = i < total ? SY[i] : INF;
-        const bool keep = v < newcap;
-        const unsigned long long incl = block_incl_scan(keep ? 1ull : 0ull, sh.tmp64, &tot);
-        if (keep) SY[kept + (uint32_t)incl - 1u] = v;
+    for (uint32_t b = 0; b < total; b += NT * kPer) {
+        const uint32_t i0 = b + tid * kPer;
+        uint32_t v[kPer];
+        uint32_t cnt = 0;
+#pragma unroll
+        for (uint32_t k = 0; k < kPer; ++k) {
+            v[k] = (i0 + k < total) ? SY[i0 + k] : INF;
+            cnt += v[k] < newcap ? 1u : 0u;
+        }
+        const unsigned long long incl = block_incl_scan((unsigned long long)cnt, sh.tmp64, &tot);
+        uint32_t o = kept + (uint32_t)incl - cnt;
+#pragma unroll
+        for (uint32_t k = 0; k < kPer; ++k)
+            if (v[k] < newcap) SY[o++] = v[k];
         kept += (uint32_t)tot;
     }
     __syncthreads();
