@@ -2,6 +2,7 @@
 (tolerance 0: the path performs no floating-point arithmetic)."""
 from __future__ import annotations
 
+import os
 from pathlib import Path
 
 import numpy as np
@@ -374,6 +375,44 @@ def test_full_size_configs(env, name, steps, over):
         assert s["n_rebalance"] > 0
     if name == "agentic_burst":
         assert s["relocated_blocks"] > 100
+
+
+_FULL_SCALE = 1_000_000 if os.environ.get("AVMP_FULL_SCALE") else 60_000
+
+
+@pytest.mark.parametrize("name,over,n_requests,max_steps", [
+    ("short_uniform", dict(seed=0), None, None),
+    ("short_uniform", dict(seed=1), None, None),
+    ("short_uniform", dict(seed=2), None, None),
+    ("mixed_long", dict(migration_batch_size=16), None, None),
+    ("mixed_long", dict(migration_batch_size=64), None, None),
+    ("agentic_burst", {}, None, 20_000),
+    ("scale", {}, _FULL_SCALE, None),
+    ("scale", dict(split=0.9, migration_enabled=False), 30_000, None),
+])
+def test_full_traces_allocator_only(env, name, over, n_requests, max_steps):
+    """The whole trace of every configuration (config 5: its first 60 000 requests unless
+    AVMP_FULL_SCALE is set), allocator only: every status of every step, the counters every 512
+    steps, every table at the end."""
+    w = W.config(name, **over)
+    g, o = _pair(env, w)
+    d = W.ClosedLoopDriver(w, requests=W.make_requests(w, n_requests) if n_requests else None)
+
+    def step(ops):
+        so = o.step(ops)
+        sg = g.step(ops)
+        assert np.array_equal(sg, so), f"statuses differ at step {d.step}"
+        if d.step % 512 == 0:
+            gs, os_ = g.stats(), o.stats()
+            assert all(gs[k] == v for k, v in os_.items()), f"counters differ at step {d.step}"
+        return so
+
+    W.record_trace(w, step, max_steps=max_steps, driver=d)
+    env["same"](g, o, w, "end of trace")
+    s = g.stats()
+    assert s["error_code"] == 0 and s["op_counter"] > 1_000_000
+    if max_steps is None:
+        assert d.done and s["free_kv"] == s["cap_kv"] and s["free_ssm"] == s["cap_ssm"]   # everything was returned
 
 
 @pytest.mark.parametrize("split,enabled", [(0.5, True), (0.5, False), (0.9, False)])
