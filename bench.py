@@ -11,7 +11,7 @@ split 0.5, B = 128, step batch 256), synthetic and seeded.  The trace is produce
 loop against the library itself (untimed), then replayed from device-resident op batches
 for the timed region.  Inputs exceed L2: every step reads and writes several GB.
 
-Prints ONE JSON line (see README for the fields).
+Prints ONE JSON line: headline value, roofline of the dominant kernel, end-to-end figure, CPU baseline.
 """
 from __future__ import annotations
 
