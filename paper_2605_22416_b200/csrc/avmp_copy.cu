@@ -19,6 +19,12 @@
 //     by the compiler's scheduling.  Every wait is bounded: a warp that gives up records
 //     AVMP_DEV_TIMEOUT and stops issuing.
 //   * generic path: plain loads and stores, for shapes whose runs are not 16-byte multiples.
+//
+// Measured alternatives that did not beat this (B200, 244 MB and 6.8 GB launches): the same walk
+// with register-staged 16-byte loads / stores at 2-8 CTAs per SM (equal within 1 %); stages of
+// 4 to 64 KiB and rings of 2 to 8 stages (equal or worse); a global ticket counter (worse);
+// staggered warp starts (worse).  The ceiling is DRAM efficiency for this read/write mix, about
+// 72-75 % of the raw rate, against 78-80 % for one long linear copy.
 #include "avmp_dev.cuh"
 
 namespace avmp {
