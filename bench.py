@@ -367,7 +367,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
         "paper_context": "the paper (pure-Python prototype, one RTX 3060 12GB) reports 1.83-13.3x goodput and a 7.6 % "
                          "OOM reduction for dynamic rebalancing against its best static baseline; it reports no "
                          "allocator ops/s, GB/s or kernel timings, so vs_baseline is null",
-        "replay_matches_closed_loop": all(st_b[k] == stats_a[k] for k in stats_a if not k.startswith("relocation_ns")),
+        "replay_matches_closed_loop": all(st_b[k] == stats_a[k] for k in stats_a if not k.startswith(("relocation_ns", "step_ns"))),
     }
     return out
 
@@ -461,7 +461,10 @@ def device_closed_loop(dev, workload: str, steps: int = 3000) -> dict:
                       "ops": st["op_counter"], "device_ms": ms, "us_per_step": ms * 1e3 / steps,
                       "ops_per_s": st["op_counter"] / (ms * 1e-3),
                       "completed_per_s_allocator_only": ds["completed"] / (ms * 1e-3),
-                      "relocation_ms": st["relocation_ns_total"] / 1e6}
+                      "relocation_ms": st["relocation_ns_total"] / 1e6,
+                      "allocator_kernel_ms": st["step_ns_total"] / 1e6,
+                      "oom_retry_share_of_allocator_kernel": st["step_ns_oom_retry"] / max(st["step_ns_total"], 1),
+                      "migration_plan_share_of_allocator_kernel": st["step_ns_migration_plan"] / max(st["step_ns_total"], 1)}
         dd.close()
         ctx.close()
     out["completed_ratio_dynamic_over_static"] = out["dynamic"]["completed"] / max(out["static"]["completed"], 1)

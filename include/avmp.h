@@ -139,6 +139,10 @@ typedef struct {
     uint64_t error_count;         /* items skipped because of device-side errors */
     uint64_t relocation_ns_last;  /* device-clock duration of the last relocation copy (first CTA in, last out) */
     uint64_t relocation_ns_total; /* sum over all relocation copies: the time spent migrating payload */
+    /* Time decomposition of the allocator kernel (paper Section 4.3), SM cycles at the nominal clock:
+     * everything; the part spent handling CapacityErrors that ended OOM; the part spent planning
+     * migrations.  The rest is service time. */
+    uint64_t step_ns_total, step_ns_oom_retry, step_ns_migration_plan;
 } avmp_stats;
 #define AVMP_N_STATS (sizeof(avmp_stats) / sizeof(uint64_t))
 

@@ -27,6 +27,7 @@ STAT_FIELDS = (
     "cap_kv", "cap_ssm", "free_kv", "free_ssm", "fsm_state", "n_invalid",
     "unit_bytes_kv", "unit_bytes_ssm", "vid_space_kv", "vid_space_ssm", "pool_bytes_aligned",
     "error_code", "error_count", "relocation_ns_last", "relocation_ns_total",
+    "step_ns_total", "step_ns_oom_retry", "step_ns_migration_plan",
 )
 
 

@@ -77,6 +77,10 @@ void fill_stats(const avmp_ctx *c, const DevState &d, avmp_stats *o)
     const uint64_t last = (d.reloc_t1 > d.reloc_t0 && d.reloc_t0 != kNone64) ? d.reloc_t1 - d.reloc_t0 : 0;
     o->relocation_ns_last = last;
     o->relocation_ns_total = d.reloc_ns_total + (d.reloc_pending ? last : 0);
+    const double ns_per_cycle = c->sm_khz > 0 ? 1e6 / (double)c->sm_khz : 0.0;
+    o->step_ns_total = (uint64_t)(d.cyc_total * ns_per_cycle);
+    o->step_ns_oom_retry = (uint64_t)(d.cyc_oom * ns_per_cycle);
+    o->step_ns_migration_plan = (uint64_t)(d.cyc_mig * ns_per_cycle);
 }
 
 }  // namespace
@@ -148,7 +152,8 @@ int avmp_create(avmp_ctx **out, const avmp_model_spec *spec, void *d_arena, uint
     int &dev = c->device;
     dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+        cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&c->sm_khz, cudaDevAttrClockRate, dev) != cudaSuccess) {
         delete c;
         return AVMP_ECUDA;
     }

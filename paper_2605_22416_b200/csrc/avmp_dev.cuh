@@ -21,6 +21,7 @@ struct DevState {
     unsigned long long migrated_bytes, wasted_bytes, relocated_blocks, relocated_bytes, gap_bytes;
     unsigned long long n_invalid, error_code, error_count;
     unsigned long long reloc_t0, reloc_t1, reloc_ns_total;   // device clock around relocation copies
+    unsigned long long cyc_total, cyc_oom, cyc_mig;          // SM cycles of the step kernel, by bucket
     uint32_t cap[2], n_free[2], n_vfree[2], fsm;
     uint32_t resume_idx;     // ops of the batch in flight already applied (multi-round steps)
     uint32_t n_reloc;        // relocation list of the last round
@@ -178,6 +179,7 @@ struct avmp_ctx {
     uint32_t B;
     int n_sms;
     int device;
+    int sm_khz;          // nominal SM clock, to turn the step kernel's cycle counts into time
     uint64_t launches;
     // staging for avmp_step_host, inside the workspace
     avmp_op *d_stage_ops;

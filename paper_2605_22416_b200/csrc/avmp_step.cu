@@ -30,6 +30,8 @@ enum : uint8_t { DIR_NONE = 0, DIR_NOP = 1, DIR_ALLOC = 2, DIR_FREE = 3 };
 struct Scalars {
     unsigned long long last, n_oom, n_ce, n_reb, migrated, wasted, reloc_blocks, reloc_bytes, gap, n_invalid;
     unsigned long long counter_base;   // logical counter before the first op of this launch
+    long long t_start, t_fail;         // SM clock: launch start, start of the failure being handled
+    unsigned long long cyc_oom, cyc_mig;
     uint32_t cap[2], nfree[2], nvfree[2], fsm;
     uint32_t migs_done, abort, abort_idx, n_reloc, reloc_pool;
     // decision of the handler in flight
@@ -215,6 +217,7 @@ step_kernel(const Geom g, const avmp_op *__restrict__ ops, const uint32_t n_ops_
         sc.n_reb = ds->n_rebalance; sc.migrated = ds->migrated_bytes; sc.wasted = ds->wasted_bytes;
         sc.reloc_blocks = ds->relocated_blocks; sc.reloc_bytes = ds->relocated_bytes;
         sc.gap = ds->gap_bytes; sc.n_invalid = ds->n_invalid; sc.counter_base = ds->op_counter;
+        sc.t_start = clock64(); sc.cyc_oom = 0; sc.cyc_mig = 0;
         for (int p = 0; p < 2; ++p) { sc.cap[p] = ds->cap[p]; sc.nfree[p] = ds->n_free[p]; sc.nvfree[p] = ds->n_vfree[p]; }
         sc.fsm = ds->fsm;
         if (ds->reloc_pending) {            // fold the last relocation copy's duration into the total
@@ -405,6 +408,8 @@ step_kernel(const Geom g, const avmp_op *__restrict__ ops, const uint32_t n_ops_
                         __syncthreads();
                         break;
                     }
+                    const uint32_t migs_before = sc.migs_done;
+                    if (tid == 0) sc.t_fail = clock64();
                     if (wantA) capacity_error(g, sh, AVMP_POOL_SSM, counter);
                     if (need_k > sc.nfree[0]) capacity_error(g, sh, AVMP_POOL_KV, counter);
                     const bool fits = need_s <= sc.nfree[1] && need_k <= sc.nfree[0];
@@ -419,6 +424,12 @@ step_kernel(const Geom g, const avmp_op *__restrict__ ops, const uint32_t n_ops_
                     } else {
                         if (tid == (int)f) { st = AVMP_ST_OOM; sc.n_oom += 1; }
                         __syncthreads();
+                    }
+                    // time decomposition (paper Section 4.3): cycles spent on this failure go to the
+                    // migration bucket if it migrated, to the OOM-retry bucket otherwise
+                    if (tid == 0) {
+                        const unsigned long long dt = (unsigned long long)(clock64() - sc.t_fail);
+                        if (sc.migs_done != migs_before) sc.cyc_mig += dt; else sc.cyc_oom += dt;
                     }
                     c2 = f + 1;
                 }
@@ -445,6 +456,9 @@ step_kernel(const Geom g, const avmp_op *__restrict__ ops, const uint32_t n_ops_
         for (int p = 0; p < 2; ++p) { ds->cap[p] = sc.cap[p]; ds->n_free[p] = sc.nfree[p]; ds->n_vfree[p] = sc.nvfree[p]; }
         ds->fsm = sc.fsm;
         ds->resume_idx = done_upto;
+        ds->cyc_total += (unsigned long long)(clock64() - sc.t_start);
+        ds->cyc_oom += sc.cyc_oom;
+        ds->cyc_mig += sc.cyc_mig;
         ds->n_reloc = sc.n_reloc;
         ds->reloc_pool = sc.reloc_pool;
         if (sc.n_reloc) { ds->reloc_t0 = kNone64; ds->reloc_t1 = 0; ds->reloc_pending = 1; }

@@ -34,7 +34,10 @@ def run_cell(w: W.Workload, step_fn: Callable[[np.ndarray], np.ndarray], stats_f
         "dynamic": bool(w.migration_enabled), "steps": d.step, "ops": s["op_counter"], "n_oom": s["n_oom"],
         "rebalances": s["n_rebalance"], "migrated_mib": s["migrated_bytes"] / W.MiB,
         "relocated_mib": s["relocated_bytes"] / W.MiB, "wasted_kib": s["wasted_bytes"] / 1024,
-        "relocation_ms": s.get("relocation_ns_total", 0) / 1e6, "completed": d.completed,
+        "relocation_ms": s.get("relocation_ns_total", 0) / 1e6,
+        "oom_retry_share": s.get("step_ns_oom_retry", 0) / max(s.get("step_ns_total", 0), 1),
+        "migration_plan_share": s.get("step_ns_migration_plan", 0) / max(s.get("step_ns_total", 0), 1),
+        "completed": d.completed,
         "preempted": d.preempted, "cap_kv": s["cap_kv"], "cap_ssm": s["cap_ssm"],
     }
 
@@ -65,7 +68,7 @@ def gpu_cell(w: W.Workload, steps: int, device="cuda:0") -> Dict:
 
 def to_markdown(rows: List[Dict]) -> str:
     cols = ("dynamic", "B", "th_low", "th_high", "n_oom", "rebalances", "migrated_mib", "relocated_mib",
-            "relocation_ms", "completed", "preempted", "cap_kv", "cap_ssm")
+            "relocation_ms", "oom_retry_share", "migration_plan_share", "completed", "preempted", "cap_kv", "cap_ssm")
     lines = ["| " + " | ".join(cols) + " |", "|" + "---|" * len(cols)]
     for r in rows:
         lines.append("| " + " | ".join(f"{r[c]:.2f}" if isinstance(r[c], float) else str(r[c]) for c in cols) + " |")
