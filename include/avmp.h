@@ -275,6 +275,15 @@ AVMP_API int avmp_gather_kv_static(avmp_ctx *ctx, uint32_t attn_layer, const uin
                                    void *d_out_k, void *d_out_v, uint64_t out_capacity_tokens,
                                    uint32_t *d_cu_seqlens, void *stream);
 
+/* Write side for a range of layers in one launch (layer first_layer + l reads its rows from the
+ * buffers advanced by l * stride bytes; rows of a layer are laid out as for the single-layer call). */
+AVMP_API int avmp_scatter_kv_layers(avmp_ctx *ctx, uint32_t first_layer, uint32_t n_layers, const uint32_t *d_reqs,
+                                    const uint32_t *d_tok_start, uint32_t n_reqs, const void *d_in_k,
+                                    const void *d_in_v, uint64_t layer_stride_bytes, void *stream);
+AVMP_API int avmp_scatter_ssm_layers(avmp_ctx *ctx, uint32_t first_layer, uint32_t n_layers, const uint32_t *d_reqs,
+                                     uint32_t n_reqs, const void *d_in_state, uint64_t state_layer_stride_bytes,
+                                     const void *d_in_conv, uint64_t conv_layer_stride_bytes, void *stream);
+
 /* Counters -> host.  Synchronises the stream. */
 AVMP_API int avmp_get_stats(avmp_ctx *ctx, avmp_stats *h_out, void *stream);
 /* Clear the sticky device error code and count.  Stream-ordered. */

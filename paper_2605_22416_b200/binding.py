@@ -100,6 +100,8 @@ def _load():
         "avmp_gather_ssm_layers": (C.c_int, [vp, C.c_uint32, C.c_uint32, vp, C.c_uint32, vp, C.c_uint64, vp, C.c_uint64, vp]),
         "avmp_scatter_kv": (C.c_int, [vp, C.c_uint32, vp, vp, C.c_uint32, vp, vp, vp]),
         "avmp_scatter_ssm": (C.c_int, [vp, C.c_uint32, vp, C.c_uint32, vp, vp, vp]),
+        "avmp_scatter_kv_layers": (C.c_int, [vp, C.c_uint32, C.c_uint32, vp, vp, C.c_uint32, vp, vp, C.c_uint64, vp]),
+        "avmp_scatter_ssm_layers": (C.c_int, [vp, C.c_uint32, C.c_uint32, vp, C.c_uint32, vp, C.c_uint64, vp, C.c_uint64, vp]),
         "avmp_get_stats": (C.c_int, [vp, C.POINTER(avmp_stats), vp]),
         "avmp_clear_error": (C.c_int, [vp, vp]),
         "avmp_export_tables": (C.c_int, [vp, C.POINTER(avmp_tables), vp]),
@@ -270,6 +272,20 @@ def avmp_scatter_ssm(ctx, ssm_layer, d_reqs, n_reqs, d_in_state, d_in_conv, stre
                                 _stream(stream)), "avmp_scatter_ssm")
 
 
+def avmp_scatter_kv_layers(ctx, first_layer, n_layers, d_reqs, d_tok_start, n_reqs, d_in_k, d_in_v, layer_stride_bytes,
+                           stream=None):
+    _check(lib.avmp_scatter_kv_layers(ctx, first_layer, n_layers, _ptr(d_reqs), _ptr(d_tok_start), n_reqs,
+                                      _ptr(d_in_k), _ptr(d_in_v), layer_stride_bytes, _stream(stream)),
+           "avmp_scatter_kv_layers")
+
+
+def avmp_scatter_ssm_layers(ctx, first_layer, n_layers, d_reqs, n_reqs, d_in_state, state_layer_stride_bytes,
+                            d_in_conv, conv_layer_stride_bytes, stream=None):
+    _check(lib.avmp_scatter_ssm_layers(ctx, first_layer, n_layers, _ptr(d_reqs), n_reqs, _ptr(d_in_state),
+                                       state_layer_stride_bytes, _ptr(d_in_conv), conv_layer_stride_bytes,
+                                       _stream(stream)), "avmp_scatter_ssm_layers")
+
+
 def avmp_get_stats(ctx, stream=None) -> dict:
     s = avmp_stats()
     _check(lib.avmp_get_stats(ctx, C.byref(s), _stream(stream)), "avmp_get_stats")
@@ -416,6 +432,15 @@ class Context:
 
     def scatter_kv(self, layer, d_reqs, d_tok_start, n, d_in_k, d_in_v, stream=None):
         avmp_scatter_kv(self.handle, layer, d_reqs, d_tok_start, n, d_in_k, d_in_v, stream)
+
+    def scatter_kv_layers(self, first_layer, n_layers, d_reqs, d_tok_start, n, d_in_k, d_in_v, layer_stride, stream=None):
+        avmp_scatter_kv_layers(self.handle, first_layer, n_layers, d_reqs, d_tok_start, n, d_in_k, d_in_v,
+                               layer_stride, stream)
+
+    def scatter_ssm_layers(self, first_layer, n_layers, d_reqs, n, d_in_state, state_stride, d_in_conv, conv_stride,
+                           stream=None):
+        avmp_scatter_ssm_layers(self.handle, first_layer, n_layers, d_reqs, n, d_in_state, state_stride,
+                                d_in_conv, conv_stride, stream)
 
     def scatter_ssm(self, layer, d_reqs, n, d_in_state, d_in_conv, stream=None):
         avmp_scatter_ssm(self.handle, layer, d_reqs, n, d_in_state, d_in_conv, stream)

@@ -334,6 +334,31 @@ int avmp_gather_ssm_layers(avmp_ctx *c, uint32_t first_layer, uint32_t n_layers,
                          d_out_conv, conv_layer_stride_bytes, L(c, stream)));
 }
 
+int avmp_scatter_kv_layers(avmp_ctx *c, uint32_t first_layer, uint32_t n_layers, const uint32_t *d_reqs,
+                           const uint32_t *d_tok_start, uint32_t n, const void *d_in_k, const void *d_in_v,
+                           uint64_t layer_stride_bytes, void *stream)
+{
+    if (!c || n_layers == 0 || (uint64_t)first_layer + n_layers > c->spec.n_attn_layers || n > c->opt.max_requests) return AVMP_EINVAL;
+    if (n == 0) return AVMP_OK;
+    if (!d_reqs || !d_in_k || !d_in_v || (((uintptr_t)d_in_k | (uintptr_t)d_in_v | layer_stride_bytes) & 15)) return AVMP_EINVAL;
+    c->launches += 2;
+    return cu(launch_kv(c->g, true, first_layer, n_layers, d_reqs, d_tok_start, n, const_cast<void *>(d_in_k),
+                        const_cast<void *>(d_in_v), layer_stride_bytes, ~0ull, nullptr, L(c, stream)));
+}
+
+int avmp_scatter_ssm_layers(avmp_ctx *c, uint32_t first_layer, uint32_t n_layers, const uint32_t *d_reqs, uint32_t n,
+                            const void *d_in_state, uint64_t state_layer_stride_bytes, const void *d_in_conv,
+                            uint64_t conv_layer_stride_bytes, void *stream)
+{
+    if (!c || n_layers == 0 || (uint64_t)first_layer + n_layers > c->spec.n_ssm_layers) return AVMP_EINVAL;
+    if (n == 0) return AVMP_OK;
+    if (!d_reqs || !d_in_state || !d_in_conv) return AVMP_EINVAL;
+    if (((uintptr_t)d_in_state | (uintptr_t)d_in_conv | state_layer_stride_bytes | conv_layer_stride_bytes) & 15) return AVMP_EINVAL;
+    c->launches += 1;
+    return cu(launch_ssm(c->g, true, first_layer, n_layers, d_reqs, n, const_cast<void *>(d_in_state),
+                         state_layer_stride_bytes, const_cast<void *>(d_in_conv), conv_layer_stride_bytes, L(c, stream)));
+}
+
 int avmp_get_stats(avmp_ctx *c, avmp_stats *h_out, void *stream)
 {
     if (!c || !h_out) return AVMP_EINVAL;

@@ -350,6 +350,28 @@ def test_multi_layer_gathers(env):
         for l in range(nl):
             os_, oc, bad = o.gather_ssm(first + l, run)
             assert bad == 0 and np.array_equal(gs[l], os_) and np.array_equal(gc[l], oc)
+    # the write side for a range of layers: fresh bytes in through one launch, out through per-layer gathers
+    torch = env["torch"]
+    rng = np.random.default_rng(9)
+    reqs = torch.from_numpy(run.view(np.int32)).cuda()
+    nl = 3
+    kb = rng.integers(0, 256, (nl, tot, m.kv_row_bytes), dtype=np.uint8)
+    vb = rng.integers(0, 256, (nl, tot, m.kv_row_bytes), dtype=np.uint8)
+    g.ctx.scatter_kv_layers(1, nl, reqs, None, len(run), torch.from_numpy(kb).cuda(), torch.from_numpy(vb).cuda(),
+                            tot * m.kv_row_bytes)
+    sb = rng.integers(0, 256, (4, len(run), m.state_bytes), dtype=np.uint8)
+    cb = rng.integers(0, 256, (4, len(run), m.conv_bytes), dtype=np.uint8)
+    g.ctx.scatter_ssm_layers(6, 4, reqs, len(run), torch.from_numpy(sb).cuda(), len(run) * m.state_bytes,
+                             torch.from_numpy(cb).cuda(), len(run) * m.conv_bytes)
+    for l in range(nl):
+        gk, gv, _, bad = g.gather_kv(1 + l, run, tot)
+        assert bad == 0 and np.array_equal(gk, kb[l]) and np.array_equal(gv, vb[l])
+    for l in range(4):
+        gs, gc, bad = g.gather_ssm(6 + l, run)
+        assert bad == 0 and np.array_equal(gs, sb[l]) and np.array_equal(gc, cb[l])
+    gk, gv, _, bad = g.gather_kv(0, run, tot)                       # untouched layers keep their bytes
+    ek, ev_, _ = h.expected_kv(0, d.uid[run], d.len[run])
+    assert np.array_equal(gk, ek) and np.array_equal(gv, ev_)
     assert g.stats()["error_code"] == 0
 
 
