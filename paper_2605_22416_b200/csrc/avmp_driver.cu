@@ -12,13 +12,12 @@
 #include <cstring>
 #include <new>
 
-#include "avmp_dev.cuh"
+#include "avmp_step_body.cuh"
 
 using namespace avmp;
 
 namespace {
 
-constexpr int NT = kStepThreads;
 constexpr uint32_t FREE_ = 0, RUNNING_ = 1;
 
 struct DrvState {
@@ -45,21 +44,30 @@ __device__ __forceinline__ void put_op(avmp_op *o, uint32_t kind, uint32_t req, 
     w[0] = kind; w[1] = req; w[2] = tokens;
 }
 
-__global__ void __launch_bounds__(NT, 1) drv_init_kernel(const Drv d, const DrvState init)
+__global__ void __launch_bounds__(kStepThreads, 1) drv_init_kernel(const Drv d, const DrvState init)
 {
     pdl_prologue();
     if (threadIdx.x == 0) { *d.st = init; *d.n_ops_word = 0; }
-    for (uint32_t s = threadIdx.x; s < init.R; s += NT) {
+    for (uint32_t s = threadIdx.x; s < init.R; s += blockDim.x) {
         d.slot_state[s] = FREE_; d.slot_uid[s] = kInvalid; d.slot_len[s] = 0; d.slot_rem[s] = 0; d.slot_seq[s] = 0;
     }
 }
 
-__global__ void __launch_bounds__(NT, 1) drv_build_kernel(const Drv d)
+// Shared memory of the two scheduler passes.
+struct DrvShared {
+    unsigned long long tmp[32];
+    DrvState st;
+    uint32_t s_completed, s_ext_ok, s_ext_oom, s_pre_uid, s_pre_len, s_pre_rem, s_has_pre;
+    unsigned long long s_best;
+};
+
+// Build the next batch (whole CTA; any block size).
+__device__ void drv_build_body(const Drv &d, DrvShared &sm)
 {
-    __shared__ unsigned long long tmp[32];
-    __shared__ DrvState st;
+    unsigned long long *tmp = sm.tmp;
+    DrvState &st = sm.st;
     const int tid = threadIdx.x;
-    pdl_prologue();
+    const uint32_t NT = blockDim.x;
     if (tid == 0) st = *d.st;
     __syncthreads();
     const uint32_t R = st.R;
@@ -105,16 +113,19 @@ __global__ void __launch_bounds__(NT, 1) drv_build_kernel(const Drv d)
         d.st->front_taken = min(n_adm, st.front_count);
         *d.n_ops_word = n_fin + n_ext + n_adm;
     }
+    __syncthreads();
 }
 
-__global__ void __launch_bounds__(NT, 1) drv_feed_kernel(const Drv d)
+// Fold the statuses of the batch back into the request slots and the queue (whole CTA).
+__device__ void drv_feed_body(const Drv &d, DrvShared &sm)
 {
-    __shared__ unsigned long long tmp[32];
-    __shared__ DrvState st;
-    __shared__ uint32_t s_completed, s_ext_ok, s_ext_oom, s_pre_uid, s_pre_len, s_pre_rem, s_has_pre;
-    __shared__ unsigned long long s_best;
+    unsigned long long *tmp = sm.tmp;
+    DrvState &st = sm.st;
+    uint32_t &s_completed = sm.s_completed, &s_ext_ok = sm.s_ext_ok, &s_ext_oom = sm.s_ext_oom;
+    uint32_t &s_pre_uid = sm.s_pre_uid, &s_pre_len = sm.s_pre_len, &s_pre_rem = sm.s_pre_rem, &s_has_pre = sm.s_has_pre;
+    unsigned long long &s_best = sm.s_best;
     const int tid = threadIdx.x;
-    pdl_prologue();
+    const uint32_t NT = blockDim.x;
     if (tid == 0) {
         st = *d.st;
         s_completed = s_ext_ok = s_ext_oom = s_has_pre = 0;
@@ -217,6 +228,36 @@ __global__ void __launch_bounds__(NT, 1) drv_feed_kernel(const Drv d)
     }
 }
 
+__global__ void __launch_bounds__(kStepThreads, 1) drv_build_kernel(const Drv d)
+{
+    __shared__ DrvShared sm;
+    pdl_prologue();
+    drv_build_body(d, sm);
+}
+
+__global__ void __launch_bounds__(kStepThreads, 1) drv_feed_kernel(const Drv d)
+{
+    __shared__ DrvShared sm;
+    pdl_prologue();
+    drv_feed_body(d, sm);
+}
+
+// One engine step of the loop in one launch: build the batch, run the allocator over it, fold the
+// statuses back.  Usable when the batch can hold at most one migration (a second one would need the
+// first one's relocation copy, which is a separate wide kernel, to run in between).
+template <int NT>
+__global__ void __launch_bounds__(NT, 1) drv_fused_kernel(const Drv d, const Geom g)
+{
+    __shared__ DrvShared sm;
+    __shared__ stepimpl::Shared<NT> sh;
+    pdl_prologue();
+    drv_build_body(d, sm);
+    const uint32_t n_ops = *d.n_ops_word;
+    stepimpl::step_body<NT>(g, sh, d.ops, n_ops, d.status, 1);
+    __syncthreads();
+    drv_feed_body(d, sm);
+}
+
 }  // namespace
 
 struct avmp_driver {
@@ -286,7 +327,7 @@ AVMP_API int avmp_driver_create(avmp_driver **out, avmp_ctx *ctx, const uint32_t
     memset(&init, 0, sizeof(init));
     init.window = concurrency; init.n_requests = n_requests; init.concurrency = concurrency; init.R = R;
     init.front_cap = l.front_cap; init.forced_slot = -1;
-    if (launch_pdl(drv_init_kernel, dim3(1), dim3(NT), 0, S(stream), d, init) != cudaSuccess) { delete dr; return AVMP_ECUDA; }
+    if (launch_pdl(drv_init_kernel, dim3(1), dim3(kStepThreads), 0, S(stream), d, init) != cudaSuccess) { delete dr; return AVMP_ECUDA; }
     ctx->launches += 1;
     *out = dr;
     return AVMP_OK;
@@ -301,11 +342,28 @@ AVMP_API int avmp_driver_destroy(avmp_driver *dr)
 AVMP_API int avmp_driver_step(avmp_driver *dr, void *stream)
 {
     if (!dr) return AVMP_EINVAL;
-    if (launch_pdl(drv_build_kernel, dim3(1), dim3(NT), 0, S(stream), dr->d) != cudaSuccess) return AVMP_ECUDA;
-    int rc = avmp_step_indirect(dr->ctx, dr->d.ops, dr->d.n_ops_word, dr->max_ops, dr->d.status, stream);
+    avmp_ctx *c = dr->ctx;
+    const bool mig = c->opt.migration_enabled != 0;
+    const uint64_t rounds = mig ? (uint64_t)(dr->max_ops - 1) / c->opt.min_rebalance_interval_ops + 1 : 1;
+    if (rounds == 1) {
+        // at most one migration fits in a batch: the whole step is one launch (plus the copy)
+        cudaError_t e;
+        if (dr->max_ops <= 256) e = launch_pdl(drv_fused_kernel<256>, dim3(1), dim3(256), 0, S(stream), dr->d, c->g);
+        else if (dr->max_ops <= 512) e = launch_pdl(drv_fused_kernel<512>, dim3(1), dim3(512), 0, S(stream), dr->d, c->g);
+        else e = launch_pdl(drv_fused_kernel<1024>, dim3(1), dim3(1024), 0, S(stream), dr->d, c->g);
+        if (e != cudaSuccess) return AVMP_ECUDA;
+        c->launches += 1;
+        if (mig) {
+            if (launch_relocate(c->g, Launch{S(stream), c->n_sms, c->device}) != cudaSuccess) return AVMP_ECUDA;
+            c->launches += 1;
+        }
+        return AVMP_OK;
+    }
+    if (launch_pdl(drv_build_kernel, dim3(1), dim3(kStepThreads), 0, S(stream), dr->d) != cudaSuccess) return AVMP_ECUDA;
+    int rc = avmp_step_indirect(c, dr->d.ops, dr->d.n_ops_word, dr->max_ops, dr->d.status, stream);
     if (rc != AVMP_OK) return rc;
-    if (launch_pdl(drv_feed_kernel, dim3(1), dim3(NT), 0, S(stream), dr->d) != cudaSuccess) return AVMP_ECUDA;
-    dr->ctx->launches += 2;
+    if (launch_pdl(drv_feed_kernel, dim3(1), dim3(kStepThreads), 0, S(stream), dr->d) != cudaSuccess) return AVMP_ECUDA;
+    c->launches += 2;
     return AVMP_OK;
 }
 
