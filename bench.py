@@ -630,7 +630,7 @@ def main():
             out["allocator"]["vs_step_batch"] = allocator_scaling(dev)
             out["closed_loop_device"] = device_closed_loop(dev, args.workload)
         if not args.no_cpu_baseline:
-            out["cpu_baseline"] = run_oracle(args, n_sample_steps=12)
+            out["cpu_baseline"] = run_oracle(args, n_sample_steps=20)
         print(json.dumps(out), flush=True)
     if world > 1:
         dist.barrier()
