@@ -279,15 +279,19 @@ def _closed_loop_parity(env, w, steps, *, with_store, kv_layers, ssm_layers, tab
             if seen["fused"] < 3 and len(d.running_slots) > 1:      # a few times per run: it moves GBs to the host
                 seen["fused"] += 1
                 _check_fused_gathers(g, h, d, w, kl, sl)
-            if with_store:
-                # the two implementations against each other, including translate of live handles
+            if len(d.running_slots):
+                # translate of every live handle of the running batch, both implementations
                 run = d.running_slots.astype(np.uint32)
                 t = o.tables()
                 handles = np.concatenate([t["req_chain"].reshape(w.max_requests, w.max_pages)[r, :t["req_npages"][r]]
                                           for r in run] + [t["req_ssm"].reshape(w.max_requests, -1)[run].reshape(-1)])
-                pg, og, bg, _ = g.translate(handles)
+                pg, og, bg, ag = g.translate(handles)
                 po, oo, bo = o.translate(handles)
                 assert bg == bo == 0 and np.array_equal(pg, po) and np.array_equal(og, oo)
+                # placement in the arena: KV units from the base up, SSM units from the end down
+                st_ = o.stats()
+                expect = np.where(po == 0, oo, np.uint64(st_["pool_bytes_aligned"] - st_["unit_bytes_ssm"]) - oo)
+                assert np.array_equal(ag, expect)
 
     W.record_trace(w, step, max_steps=steps, driver=d, on_step=on_step)
     env["same"](g, o, w, "end")
