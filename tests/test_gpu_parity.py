@@ -383,11 +383,11 @@ def test_multi_layer_gathers(env):
     ("short_uniform", 1200, {}),
     ("short_uniform", 500, dict(seed=1)),
     ("short_uniform", 500, dict(seed=2, migration_enabled=False)),
-    ("mixed_long", 1200, dict(migration_batch_size=4)),
-    ("mixed_long", 1200, dict(migration_batch_size=16)),
-    ("mixed_long", 1200, dict(migration_batch_size=64)),
+    ("mixed_long", 700, dict(migration_batch_size=4)),
+    ("mixed_long", 700, dict(migration_batch_size=16)),
+    ("mixed_long", 700, dict(migration_batch_size=64)),
     ("mixed_long", 150, dict(migration_batch_size=16, split=0.1)),   # the mirrored reading of "split"
-    ("agentic_burst", 1500, {}),
+    ("agentic_burst", 900, {}),
 ])
 def test_full_size_configs(env, name, steps, over):
     """Configs 2-4 at their full pool sizes and step batches: statuses and counters every
@@ -445,9 +445,9 @@ def test_full_traces_allocator_only(env, name, over, n_requests, max_steps):
 def test_scale_config(env, split, enabled):
     """Config 5: 72-layer model, 120 GiB pool resident in HBM, step batch 1024."""
     w = W.config("scale", split=split, migration_enabled=enabled)
-    s, seen, d = _closed_loop_parity(env, w, 120 if enabled else 60, with_store=False, kv_layers=[4],
+    s, seen, d = _closed_loop_parity(env, w, 80 if enabled else 50, with_store=False, kv_layers=[4],
                                      ssm_layers=[31], table_every=40, gather_every=59, max_migration_checks=6)
-    assert seen["tokens"] > 0 and s["op_counter"] > 40_000
+    assert seen["tokens"] > 0 and s["op_counter"] > 30_000
 
 
 def test_sensitivity_sweep_cells_match_the_oracle(env):
