@@ -23,7 +23,8 @@
 // Measured alternatives that did not beat this (B200, 244 MB and 6.8 GB launches): the same walk
 // with register-staged 16-byte loads / stores at 2-8 CTAs per SM (equal within 1 %); stages of
 // 4 to 64 KiB and rings of 2 to 8 stages (equal or worse); a global ticket counter (worse);
-// staggered warp starts (worse).  The ceiling is DRAM efficiency for this read/write mix, about
+// staggered warp starts (worse); smaller pieces for small launches, to even out the last round
+// of the walk (worse: small launches are bound by ramp and tail latency, not by imbalance).  The ceiling is DRAM efficiency for this read/write mix, about
 // 72-75 % of the raw rate, against 78-80 % for one long linear copy.
 #include "avmp_dev.cuh"
 
