@@ -446,7 +446,7 @@ def test_scale_config(env, split, enabled):
     """Config 5: 72-layer model, 120 GiB pool resident in HBM, step batch 1024."""
     w = W.config("scale", split=split, migration_enabled=enabled)
     s, seen, d = _closed_loop_parity(env, w, 80 if enabled else 50, with_store=False, kv_layers=[4],
-                                     ssm_layers=[31], table_every=40, gather_every=59, max_migration_checks=6)
+                                     ssm_layers=[31], table_every=25, gather_every=23, max_migration_checks=6)
     assert seen["tokens"] > 0 and s["op_counter"] > 30_000
 
 
