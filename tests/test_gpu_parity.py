@@ -582,6 +582,18 @@ def test_edge_cases(env):
     env["same"](g, o, w, "after step_host")
 
 
+def test_both_pools_short_in_one_op(env):
+    """An admit short in both pools: SSM handler first (migrates), then the KV handler (throttled)."""
+    w = W.config("tiny", pool_bytes=2048, migration_batch_size=3)
+    g, o = _pair(env, w, max_requests=12, max_pages=8)
+    ops = np.concatenate([W.make_ops(W.OP_ADMIT, np.arange(10), 1), W.make_ops(W.OP_ADMIT, [10], 96)])
+    sg, so = g.step(ops), o.step(ops)
+    assert np.array_equal(sg, so) and so[-1] == W.ST_OOM
+    s = g.stats()
+    assert (s["n_capacity_error"], s["n_rebalance"], s["cap_kv"], s["free_kv"], s["cap_ssm"], s["free_ssm"]) == (2, 1, 13, 3, 12, 2)
+    env["same"](g, o, w, "both short")
+
+
 def test_create_rejects_bad_configurations(env):
     from paper_2605_22416_b200 import binding as B
     torch = env["torch"]

@@ -337,6 +337,55 @@ def test_no_donor_means_static_behaviour():
     assert s["fsm_state"] == 1      # KV free fraction 0 < threshold_low: KV_PRESSURED
 
 
+def test_ssm_shortage_is_handled_before_kv_shortage():
+    """Group allocation checks the SSM pool first.  Worked by hand: 16 KV pages / 10 SSM blocks,
+    B = 3.  Ten one-page requests fill the SSM store (KV: 6 of 16 free = 0.375).  An admit that
+    needs 1 block and exactly the 6 free pages raises CapacityError(SSM); KV donates 3 pages
+    (192 B -> 2 blocks); now only 3 pages are free, so the same op raises CapacityError(KV), which
+    the throttle keeps from migrating: OOM after two handler runs and one migration.  (Checking KV
+    first would see 6 <= 6, run one handler only, and still end OOM.)"""
+    w = W.config("tiny", pool_bytes=2048, migration_batch_size=3)
+    o = Oracle.from_workload(w, max_requests=12, max_pages=8)
+    assert (o.step(W.make_ops(W.OP_ADMIT, np.arange(10), 1)) == 0).all()
+    s = o.stats()
+    assert (s["free_kv"], s["free_ssm"]) == (6, 0)
+    st = o.step(W.make_ops(W.OP_ADMIT, [10], 96))
+    s = o.stats()
+    assert int(st[0]) == W.ST_OOM
+    assert (s["n_capacity_error"], s["n_rebalance"], s["n_oom"]) == (2, 1, 1)
+    assert (s["cap_kv"], s["free_kv"], s["cap_ssm"], s["free_ssm"]) == (13, 3, 12, 2)
+    assert s["migrated_bytes"] == 192 and s["wasted_bytes"] == 0 and s["last_rebalance_op"] == 11
+
+
+def test_threshold_comparisons_are_strict():
+    """Section 3.2: the donor must have a free fraction *greater than* threshold_high.  With exactly
+    0.30 free (3 of 10 blocks) nothing migrates; with 0.40 (4 of 10) it does."""
+    w = W.config("tiny", pool_bytes=2048, migration_batch_size=2)          # 16 KV pages, 10 SSM blocks
+    for n_req, tokens, migrates in ((7, [48, 48, 32, 32, 32, 32, 32], False), (6, [48, 48, 48, 48, 32, 32], True)):
+        o = Oracle.from_workload(w, max_requests=8, max_pages=8)
+        s0 = o.stats()
+        assert (s0["cap_kv"], s0["cap_ssm"]) == (16, 10)
+        assert (o.step(W.make_ops(W.OP_ADMIT, np.arange(n_req), tokens)) == 0).all()
+        s = o.stats()
+        assert s["free_kv"] == 0 and s["free_ssm"] == 10 - n_req
+        st = o.step(W.make_ops(W.OP_EXTEND, [0], 1))
+        s = o.stats()
+        assert s["n_capacity_error"] == 1
+        assert (s["n_rebalance"] == 1) == migrates and int(st[0]) == (W.ST_OK if migrates else W.ST_OOM)
+    # threshold_low labels the state only when the free fraction is *below* it: 1 free of 20 is exactly 0.05
+    m = W.ModelShape(1, 1, 16, 1, 1, 2, 20, 4, 4)
+    o = Oracle(m, 1536, 256 / 1536, 1, max_requests=4, max_pages=32, migration_enabled=False)   # 1280 B KV + 256 B SSM
+    s0 = o.stats()
+    assert s0["cap_kv"] == 20, s0
+    o.step(W.make_ops(W.OP_ADMIT, [0], 19 * 16))
+    st = o.step(W.make_ops(W.OP_ADMIT, [1], 2 * 16))       # needs 2 pages, 1 free: CapacityError(KV)
+    s = o.stats()
+    assert int(st[0]) == W.ST_OOM and s["free_kv"] == 1 and s["fsm_state"] == 0      # 0.05 is not < 0.05
+    o.step(W.make_ops(W.OP_EXTEND, [0], 16))                # takes the last page
+    o.step(W.make_ops(W.OP_EXTEND, [0], 16))                # CapacityError at 0 free: now pressured
+    assert o.stats()["fsm_state"] == 1
+
+
 # ---- threshold_low null result (Section 4.5, stage 2) and determinism (Section 4.1) ------
 def _digest(o: Oracle):
     import hashlib
