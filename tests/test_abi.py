@@ -30,6 +30,23 @@ def test_library_exports_every_declared_symbol():
         assert hasattr(lib, name), f"{name} is declared in avmp.h but not exported"
 
 
+def test_public_header_is_plain_c():
+    """The boundary is a C ABI: avmp.h must compile as C99 (and as C++) on its own."""
+    hdr = str(ROOT / "include" / "avmp.h")
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only", "-x", "c", hdr])
+    subprocess.check_call(["g++", "-std=c++14", "-Wall", "-Werror", "-fsyntax-only", "-x", "c++", hdr])
+    # and a C program can link against the library without any CUDA header
+    src = ROOT / "tests" / "c_abi_smoke.c"
+    from paper_2605_22416_b200 import build
+    lib = build.build_library()
+    exe = Path(os.environ.get("TMPDIR", "/tmp")) / f"avmp_c_abi_smoke_{os.getpid()}"
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", f"-I{ROOT / 'include'}", str(src), "-o", str(exe),
+                           str(lib), f"-Wl,-rpath,{lib.parent}"])
+    out = subprocess.check_output([str(exe)]).decode()
+    exe.unlink()
+    assert "U_kv=262144 U_ssm=622592 kv_cap=8192 ssm_cap=3449" in out and "workspace_bytes=" in out
+
+
 def test_binding_declares_every_symbol():
     src = (ROOT / "paper_2605_22416_b200" / "binding.py").read_text()
     header = (ROOT / "include" / "avmp.h").read_text()
