@@ -474,6 +474,62 @@ def device_closed_loop(dev, workload: str, steps: int = 3000) -> dict:
     return out
 
 
+def write_side_microbench(dev) -> dict:
+    """The write side and translate on their own: all-layer scatters of the same shapes the gathers
+    move, and a million handle translations."""
+    import torch
+    from paper_2605_22416_b200 import binding as B
+    m = W.JAMBA_LIKE
+    ctx = B.Context(m, 8 * W.GiB, 0.6, 128, max_requests=256, max_pages=256, device=dev)
+    n, tokens = 96, 2048
+    st = np.zeros(n, np.uint32)
+    ctx.step_host(W.make_ops(W.OP_ADMIT, np.arange(n), tokens), n, st)
+    assert (st == 0).all()
+    reqs = torch.arange(n, dtype=torch.int32, device=dev)
+    tot = n * tokens
+    kb = torch.empty((m.n_attn_layers, tot, m.kv_row_bytes), dtype=torch.uint8, device=dev)
+    vb = torch.empty((m.n_attn_layers, tot, m.kv_row_bytes), dtype=torch.uint8, device=dev)
+    sb = torch.empty((m.n_ssm_layers, n, m.state_bytes), dtype=torch.uint8, device=dev)
+    cb = torch.empty((m.n_ssm_layers, n, m.conv_bytes), dtype=torch.uint8, device=dev)
+    sid = torch.cuda.current_stream().cuda_stream
+    peak, _ = _peaks()
+
+    def timed(fn, reps=5):
+        fn()
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize(dev)
+        return e0.elapsed_time(e1) / reps
+
+    kv_bytes = 2 * tot * 2 * m.kv_row_bytes * m.n_attn_layers
+    ssm_bytes = 2 * n * (m.state_bytes + m.conv_bytes) * m.n_ssm_layers
+    ms_kv = timed(lambda: ctx.scatter_kv_layers(0, m.n_attn_layers, reqs, None, n, kb, vb, tot * m.kv_row_bytes, sid))
+    ms_ssm = timed(lambda: ctx.scatter_ssm_layers(0, m.n_ssm_layers, reqs, n, sb, n * m.state_bytes, cb,
+                                                  n * m.conv_bytes, sid))
+    # translate: every handle of the batch, repeated to a million entries
+    t, _ = ctx.export_tables()
+    chain = t["req_chain"].reshape(256, 256)
+    handles = np.concatenate([chain[r, :t["req_npages"][r]] for r in range(n)] +
+                             [t["req_ssm"].reshape(256, m.n_ssm_layers)[:n].reshape(-1)]).astype(np.uint32)
+    handles = np.resize(handles, 1 << 20)
+    d_h = torch.from_numpy(handles.view(np.int32)).to(dev)
+    d_pool = torch.empty(len(handles), dtype=torch.int32, device=dev)
+    d_off = torch.empty(len(handles), dtype=torch.int64, device=dev)
+    d_aoff = torch.empty(len(handles), dtype=torch.int64, device=dev)
+    ms_tr = timed(lambda: ctx.translate(d_h, len(handles), d_pool, d_off, d_aoff, sid))
+    err = ctx.stats()["error_code"]
+    ctx.close()
+    return {"scatter_kv_layers_gbs": kv_bytes / (ms_kv * 1e-3) / 1e9, "scatter_kv_frac_of_peak": kv_bytes / (ms_kv * 1e-3) / 1e9 / peak,
+            "scatter_ssm_layers_gbs": ssm_bytes / (ms_ssm * 1e-3) / 1e9, "scatter_ssm_frac_of_peak": ssm_bytes / (ms_ssm * 1e-3) / 1e9 / peak,
+            "translate_handles_per_s": len(handles) / (ms_tr * 1e-3), "translate_us_per_million": ms_tr * 1e3,
+            "device_error_code": err,
+            "note": f"{n} requests x {tokens} tokens, all {m.n_attn_layers} attention / {m.n_ssm_layers} SSM layers per launch"}
+
+
 def allocator_scaling(dev, batches=(32, 256, 1024, 4096), warm=120, timed=60) -> list:
     """avmp_step alone on closed-loop traces of growing step batch (small units so that
     thousands of requests fit): the path is latency-bound, so ops/s grows with the batch."""
@@ -629,6 +685,7 @@ def main():
             out["migration"]["microbench"] = migration_microbench(dev)
             out["allocator"]["vs_step_batch"] = allocator_scaling(dev)
             out["closed_loop_device"] = device_closed_loop(dev, args.workload)
+            out["write_side"] = write_side_microbench(dev)
         if not args.no_cpu_baseline:
             out["cpu_baseline"] = run_oracle(args, n_sample_steps=20)
         print(json.dumps(out), flush=True)
