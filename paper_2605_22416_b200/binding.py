@@ -377,6 +377,7 @@ class Context:
         if ws == 0:
             raise AvmpError("avmp_workspace_bytes rejected the configuration")
         with torch.cuda.device(self.device):
+            self._owns_arena = arena is None
             self.arena = arena if arena is not None else torch.empty(pool_bytes, dtype=torch.uint8, device=self.device)
             self.workspace = torch.empty(ws, dtype=torch.uint8, device=self.device)
             self.handle = avmp_create(self.spec, self.arena, pool_bytes, initial_split, migration_batch_size,
@@ -395,6 +396,10 @@ class Context:
             torch.cuda.synchronize(self.device)
             avmp_destroy(self.handle)
             self.handle = None
+            # drop the device memory this object allocated, so that the next context fits
+            self.workspace = None
+            if self._owns_arena:
+                self.arena = None
 
     def __del__(self):
         try:
@@ -492,6 +497,7 @@ class DeviceDriver:
             torch.cuda.synchronize(self.ctx.device)
             avmp_driver_destroy(self.handle)
             self.handle = None
+            self.workspace = self.d_prompt = self.d_output = None
 
     def __del__(self):
         try:
