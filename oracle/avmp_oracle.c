@@ -167,8 +167,12 @@ static void capacity_error(orc_ctx *c, int X)
 
     uint64_t n = c->B < c->n_free[Y] ? c->B : c->n_free[Y];
     uint64_t ceded = n * c->U[Y];
-    uint64_t mgain = ceded / c->U[X];
-    uint64_t waste = ceded % c->U[X];     /* donor bytes freed modulo the recipient unit */
+    /* Section 3.2 as written: the recipient gets the whole units that fit in the ceded bytes and
+     * the remainder is wasted.  With reclaim_gap (a variant, not in the paper) the bytes already
+     * stranded between the pools are offered again together with the ceded ones. */
+    uint64_t carry = c->o.reclaim_gap ? c->gap : 0;
+    uint64_t mgain = (carry + ceded) / c->U[X];
+    uint64_t waste = (carry + ceded) % c->U[X];   /* bytes freed modulo the recipient unit */
     if (mgain == 0) return;               /* nothing whole to hand over: state untouched */
 
     c->fsm = ORC_REBALANCING;
@@ -200,8 +204,8 @@ static void capacity_error(orc_ctx *c, int X)
         c->S[X][c->n_free[X]++] = (uint32_t)s;
     c->cap[X] += (uint32_t)mgain;
 
-    c->gap += waste;
-    c->wasted_bytes += waste;
+    c->gap = c->gap - carry + waste;
+    if (!c->o.reclaim_gap) c->wasted_bytes += waste;   /* with reclaim nothing is lost for good */
     c->migrated_bytes += ceded;
     c->n_rebalance += 1;
     c->last_rebalance_op = c->op_counter;

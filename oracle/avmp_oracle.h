@@ -54,6 +54,7 @@ typedef struct {
     uint64_t min_rebalance_interval_ops;
     uint32_t migration_enabled;
     uint32_t max_requests, max_pages_per_request;
+    uint32_t reclaim_gap;   /* 0 = waste is lost to the gap (Section 3.2 as written); 1 = see capacity_error */
 } orc_options;
 
 typedef struct {

@@ -42,7 +42,8 @@ class _Model(C.Structure):
 class _Options(C.Structure):
     _fields_ = [("threshold_low_ppm", C.c_uint32), ("threshold_high_ppm", C.c_uint32),
                 ("min_rebalance_interval_ops", C.c_uint64), ("migration_enabled", C.c_uint32),
-                ("max_requests", C.c_uint32), ("max_pages_per_request", C.c_uint32)]
+                ("max_requests", C.c_uint32), ("max_pages_per_request", C.c_uint32),
+                ("reclaim_gap", C.c_uint32)]
 
 
 def build(force: bool = False) -> Path:
@@ -97,11 +98,11 @@ class Oracle:
     def __init__(self, model, pool_bytes: int, split: float, migration_batch_size: int, *,
                  max_requests: int, max_pages: int, threshold_low_ppm: int = 50_000,
                  threshold_high_ppm: int = 300_000, min_rebalance_interval_ops: int = 1000,
-                 migration_enabled: bool = True, with_store: bool = False):
+                 migration_enabled: bool = True, reclaim_gap: bool = False, with_store: bool = False):
         self.model = model
         m = _Model(*(int(getattr(model, f[0])) for f in _Model._fields_))
         o = _Options(threshold_low_ppm, threshold_high_ppm, min_rebalance_interval_ops,
-                     int(migration_enabled), max_requests, max_pages)
+                     int(migration_enabled), max_requests, max_pages, int(reclaim_gap))
         self.max_requests, self.max_pages = max_requests, max_pages
         self._h = lib().orc_create(C.byref(m), pool_bytes, float(split), migration_batch_size,
                                    C.byref(o), int(with_store))
@@ -113,7 +114,7 @@ class Oracle:
         kw = dict(max_requests=w.max_requests, max_pages=w.max_pages,
                   threshold_low_ppm=w.threshold_low_ppm, threshold_high_ppm=w.threshold_high_ppm,
                   min_rebalance_interval_ops=w.min_rebalance_interval_ops,
-                  migration_enabled=w.migration_enabled, with_store=with_store)
+                  migration_enabled=w.migration_enabled, reclaim_gap=w.reclaim_gap, with_store=with_store)
         kw.update(over)
         return cls(w.model, w.pool_bytes, w.split, w.migration_batch_size, **kw)
 

@@ -188,6 +188,7 @@ class Workload:
     n_requests: int
     seed: int = 0
     migration_enabled: bool = True
+    reclaim_gap: bool = False          # variant: gap bytes are offered again at the next migration
     min_rebalance_interval_ops: int = 1000
     threshold_low_ppm: int = 50_000
     threshold_high_ppm: int = 300_000

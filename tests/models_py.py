@@ -113,12 +113,13 @@ class CountsModel(_ReqCounts):
     the threshold_high trigger and the waste formula."""
 
     def __init__(self, model, pool_bytes, split, B, max_requests, max_pages, *, th_high_ppm=300_000,
-                 min_interval=1000, enabled=True):
+                 min_interval=1000, enabled=True, reclaim=False):
         super().__init__(model, max_requests, max_pages)
         kv, ssm, p_al = initial_caps(model, pool_bytes, split)
         self.U = list(unit_sizes(model))
         self.cap = [kv, ssm]
         self.free = [kv, ssm]
+        self.p_al, self.reclaim = p_al, reclaim
         self.B, self.th_high, self.min_interval, self.enabled = B, th_high_ppm, min_interval, enabled
         self.clock = 0
         self.last: Optional[int] = None
@@ -137,6 +138,11 @@ class CountsModel(_ReqCounts):
             return
         n = min(self.B, self.free[y])
         gain, waste = divmod(n * self.U[y], self.U[x])
+        if self.reclaim:
+            # everything between the two pools after the donor shrank is on offer (no stored gap:
+            # the middle follows from the capacities)
+            middle = self.p_al - (self.cap[y] - n) * self.U[y] - self.cap[x] * self.U[x]
+            gain, waste = middle // self.U[x], 0
         if gain == 0:
             return
         self.events.append(dict(clock=self.clock, donor=y, n=n, gain=gain, waste=waste,
@@ -192,9 +198,10 @@ class NaiveAllocator:
     index 0 -- the mirror image of an array stack).  Payload lives in `bytes_at[pool][slot]`."""
 
     def __init__(self, model, pool_bytes, split, B, max_requests, max_pages, *, th_high_ppm=300_000,
-                 min_interval=1000, enabled=True):
+                 min_interval=1000, enabled=True, reclaim=False):
         self.model = model
         kv, ssm, p_al = initial_caps(model, pool_bytes, split)
+        self.p_al, self.reclaim = p_al, reclaim
         self.U = list(unit_sizes(model))
         self.cap = [kv, ssm]
         self.next_slots = [list(range(kv)), list(range(ssm))]
@@ -232,6 +239,8 @@ class NaiveAllocator:
             return
         n = min(self.B, nfree)
         gain = n * self.U[y] // self.U[x]
+        if self.reclaim:
+            gain = (self.p_al - (self.cap[y] - n) * self.U[y] - self.cap[x] * self.U[x]) // self.U[x]
         if gain == 0:
             return
         newcap = self.cap[y] - n

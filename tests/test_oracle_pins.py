@@ -83,14 +83,15 @@ def test_translate_rejects_dead_handles():
 
 
 # ---- the hand-worked trace ------------------------------------------------------------
-def test_worked_example():
-    w = W.config("tiny")
+@pytest.mark.parametrize("golden,reclaim", [("worked_example.txt", False), ("worked_example_reclaim.txt", True)])
+def test_worked_example(golden, reclaim):
+    w = W.config("tiny", reclaim_gap=reclaim)
     o = Oracle.from_workload(w)
     kinds = {"ADMIT": 1, "EXTEND": 2, "FINISH": 3}
     cols = ("cap_kv", "free_kv", "cap_ssm", "free_ssm", "gap_bytes", "migrated_bytes", "wasted_bytes",
             "n_rebalance", "relocated_blocks", "n_oom", "n_capacity_error")
     extra = {}
-    for line in _rows("worked_example.txt"):
+    for line in _rows(golden):
         if "|" in line:
             l, r = line.split("|")
             k, req, tok = l.split()
@@ -169,6 +170,34 @@ def test_no_whole_unit_no_migration():
     s = o.stats()
     assert s["n_rebalance"] == 0 and s["n_capacity_error"] == 1 and s["last_rebalance_op"] == NONE64
     assert s["cap_kv"] == s0["cap_kv"] and s["cap_ssm"] == 28
+
+
+def test_reclaim_gap_offers_stranded_bytes_again():
+    # Variant of the waste rule: one ceded KV page (256 KiB) is less than an SSM block (608 KiB),
+    # but together with 400 000 B already lying between the pools it makes one block.
+    m = W.JAMBA_LIKE
+    u_kv, u_ssm = M.unit_sizes(m)
+    pool = 10 * u_kv + 28 * u_ssm + 400_000
+    split = (28 * u_ssm + 400_000 - 300) / pool       # the slack sits in the SSM share: no 11th page
+    for reclaim in (False, True):
+        o = Oracle(m, pool, split, 1, max_requests=4, max_pages=8, min_rebalance_interval_ops=1,
+                   reclaim_gap=reclaim)
+        s0 = o.stats()
+        assert (s0["cap_kv"], s0["cap_ssm"], s0["gap_bytes"]) == (10, 28, 400_000)
+        st = o.step(W.make_ops(W.OP_ADMIT, [0, 1], [1, 1])).tolist()
+        s = o.stats()
+        if not reclaim:
+            assert st == [W.ST_OK, W.ST_OOM] and s["n_rebalance"] == 0 and s["gap_bytes"] == 400_000
+        else:
+            # 400 000 + 262 144 = 662 144 = 1 block + 39 552: still not the 28 blocks an admit needs
+            assert st == [W.ST_OK, W.ST_OOM] and s["n_rebalance"] == 1
+            assert (s["cap_kv"], s["cap_ssm"], s["gap_bytes"]) == (9, 29, 39_552)
+            assert s["wasted_bytes"] == 0 and s["migrated_bytes"] == u_kv
+            # the second page offered meets a gap of 39 552: 301 696 B is no block, nothing happens
+            assert o.step(W.make_ops(W.OP_ADMIT, [1], [1])).tolist() == [W.ST_OOM]
+            s2 = o.stats()
+            assert s2["n_rebalance"] == 1 and s2["gap_bytes"] == 39_552 and s2["cap_kv"] == 9
+        _inv(o, W.config("short_uniform"))
 
 
 # ---- configuration validation (Section 4.6) ----------------------------------------------

@@ -23,17 +23,19 @@ shapes = st.builds(
 @settings(max_examples=60, deadline=None, suppress_health_check=[HealthCheck.too_slow])
 @given(shape=shapes, pool_units=st.integers(6, 40), split=st.sampled_from([0.0, 0.2, 0.5, 0.8, 1.0]),
        B=st.integers(1, 9), interval=st.integers(1, 12), th_high=st.sampled_from([100_000, 300_000, 600_000]),
-       seed=st.integers(0, 10_000), enabled=st.booleans())
-def test_oracle_equals_naive_and_counts_models(shape, pool_units, split, B, interval, th_high, seed, enabled):
+       seed=st.integers(0, 10_000), enabled=st.booleans(), reclaim=st.booleans())
+def test_oracle_equals_naive_and_counts_models(shape, pool_units, split, B, interval, th_high, seed, enabled,
+                                               reclaim):
     u_kv, u_ssm = M.unit_sizes(shape)
     pool = pool_units * max(u_kv, u_ssm)
     kv0, ssm0, _ = M.initial_caps(shape, pool, split)
     if kv0 == 0 and ssm0 == 0:
         return
     R, MP = 5, 6
-    kw = dict(th_high_ppm=th_high, min_interval=interval, enabled=enabled)
+    kw = dict(th_high_ppm=th_high, min_interval=interval, enabled=enabled, reclaim=reclaim)
     o = Oracle(shape, pool, split, B, max_requests=R, max_pages=MP, threshold_low_ppm=50_000,
-               threshold_high_ppm=th_high, min_rebalance_interval_ops=interval, migration_enabled=enabled)
+               threshold_high_ppm=th_high, min_rebalance_interval_ops=interval, migration_enabled=enabled,
+               reclaim_gap=reclaim)
     nv = M.NaiveAllocator(shape, pool, split, B, R, MP, **kw)
     cm = M.CountsModel(shape, pool, split, B, R, MP, **kw)
     ops = W.random_op_string(seed, 120, R, shape.page_tokens * 4, p_invalid=0.08)
