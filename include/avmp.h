@@ -94,6 +94,12 @@ typedef struct {
     uint32_t migration_enabled;           /* 0 = static partition with AVMP handles */
     uint32_t max_requests;                /* request slots: op.req is in [0, max_requests) */
     uint32_t max_pages_per_request;       /* longest KV chain, in pages */
+    uint32_t reclaim_gap;                 /* 0 (default): the paper's rule, recipient gains floor(n*U_donor /
+                                             U_recipient) units and the remainder is lost to the gap between
+                                             the pools.  1: a variant with no counterpart in the paper, the
+                                             bytes already in the gap are offered again with the ceded ones:
+                                             gain = floor((gap + n*U_donor) / U_recipient), gap = remainder,
+                                             wasted_bytes stays 0 */
 } avmp_options;
 
 /* One allocator operation, 12 bytes. */

@@ -40,7 +40,8 @@ class avmp_model_spec(C.Structure):
 class avmp_options(C.Structure):
     _fields_ = [("threshold_low_ppm", C.c_uint32), ("threshold_high_ppm", C.c_uint32),
                 ("min_rebalance_interval_ops", C.c_uint64), ("migration_enabled", C.c_uint32),
-                ("max_requests", C.c_uint32), ("max_pages_per_request", C.c_uint32)]
+                ("max_requests", C.c_uint32), ("max_pages_per_request", C.c_uint32),
+                ("reclaim_gap", C.c_uint32)]
 
 
 class avmp_layout(C.Structure):
@@ -363,14 +364,15 @@ class Context:
     def __init__(self, model, pool_bytes: int, initial_split: float, migration_batch_size: int, *,
                  max_requests: int, max_pages: int, threshold_low_ppm: int = 50_000,
                  threshold_high_ppm: int = 300_000, min_rebalance_interval_ops: int = 1000,
-                 migration_enabled: bool = True, device="cuda:0", arena: Optional[torch.Tensor] = None):
+                 migration_enabled: bool = True, reclaim_gap: bool = False, device="cuda:0",
+                 arena: Optional[torch.Tensor] = None):
         if not torch.cuda.is_available():
             raise AvmpError("AVMP needs a CUDA device; there is no CPU path")
         self.device = torch.device(device)
         self.model = model
         self.spec = model_spec(model)
         self.opt = avmp_options(threshold_low_ppm, threshold_high_ppm, min_rebalance_interval_ops,
-                                int(migration_enabled), max_requests, max_pages)
+                                int(migration_enabled), max_requests, max_pages, int(reclaim_gap))
         self.pool_bytes = pool_bytes
         self.layout = avmp_derive_layout(self.spec, pool_bytes, initial_split)
         ws = avmp_workspace_bytes(self.spec, pool_bytes, self.opt)
@@ -387,7 +389,8 @@ class Context:
     def from_workload(cls, w, **over):
         kw = dict(max_requests=w.max_requests, max_pages=w.max_pages,
                   threshold_low_ppm=w.threshold_low_ppm, threshold_high_ppm=w.threshold_high_ppm,
-                  min_rebalance_interval_ops=w.min_rebalance_interval_ops, migration_enabled=w.migration_enabled)
+                  min_rebalance_interval_ops=w.min_rebalance_interval_ops, migration_enabled=w.migration_enabled,
+                  reclaim_gap=w.reclaim_gap)
         kw.update(over)
         return cls(w.model, w.pool_bytes, w.split, w.migration_batch_size, **kw)
 

@@ -92,7 +92,7 @@ void avmp_default_options(avmp_options *o)
     if (!o) return;
     o->threshold_low_ppm = 50000; o->threshold_high_ppm = 300000;
     o->min_rebalance_interval_ops = 1000; o->migration_enabled = 1;
-    o->max_requests = 1024; o->max_pages_per_request = 4096;
+    o->max_requests = 1024; o->max_pages_per_request = 4096; o->reclaim_gap = 0;
 }
 
 int avmp_derive_layout(const avmp_model_spec *m, uint64_t pool_bytes, double split, avmp_layout *out)
@@ -167,6 +167,7 @@ int avmp_create(avmp_ctx **out, const avmp_model_spec *spec, void *d_arena, uint
     g.T = spec->page_tokens; g.na = spec->n_attn_layers; g.ns = spec->n_ssm_layers;
     g.R = o.max_requests; g.max_pages = o.max_pages_per_request; g.B = migration_batch_size;
     g.th_low = o.threshold_low_ppm; g.th_high = o.threshold_high_ppm; g.migration_enabled = o.migration_enabled;
+    g.reclaim_gap = o.reclaim_gap ? 1u : 0u;
     g.arena = static_cast<uint8_t *>(d_arena);
     g.st = reinterpret_cast<DevState *>(base + w.state);
     for (int p = 0; p < 2; ++p) {

@@ -34,7 +34,7 @@ struct DevState {
 struct Geom {
     unsigned long long P_al, U[2], kv_layer_bytes, row_bytes, state_bytes, conv_bytes, min_interval;
     uint32_t V[2];
-    uint32_t T, na, ns, R, max_pages, B, th_low, th_high, migration_enabled;
+    uint32_t T, na, ns, R, max_pages, B, th_low, th_high, migration_enabled, reclaim_gap;
     uint8_t *arena;
     DevState *st;
     uint32_t *S[2], *W[2], *VT[2], *OW[2];

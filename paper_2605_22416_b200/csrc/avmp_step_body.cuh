@@ -46,7 +46,8 @@ __device__ __forceinline__ bool would_migrate(const Geom &g, const Scalars &sc, 
     if (!((unsigned long long)sc.nfree[Y] * 1000000ull > (unsigned long long)g.th_high * sc.cap[Y])) return false;
     if (sc.last != kNone64 && counter - sc.last < g.min_interval) return false;
     const unsigned long long n = g.B < sc.nfree[Y] ? g.B : sc.nfree[Y];
-    return (n * g.U[Y]) / g.U[X] >= 1ull;
+    // reclaim_gap variant: the bytes already lying between the pools are offered again
+    return (n * g.U[Y] + (g.reclaim_gap ? sc.gap : 0ull)) / g.U[X] >= 1ull;
 }
 
 // Section 3.2 handler for a shortage in pool X at logical time `counter`; whole CTA.
@@ -66,10 +67,11 @@ __device__ void capacity_error(const Geom &g, Shared<NT> &sh, int X, unsigned lo
         sc.mig = would_migrate(g, sc, X, counter) ? 1u : 0u;
         if (sc.mig) {
             const unsigned long long n = g.B < sc.nfree[Y] ? g.B : sc.nfree[Y];
-            const unsigned long long ceded = n * g.U[Y];
+            const unsigned long long carry = g.reclaim_gap ? sc.gap : 0ull;
+            const unsigned long long avail = n * g.U[Y] + carry;
             sc.mig_n = (uint32_t)n;
-            sc.mig_m = (uint32_t)(ceded / g.U[X]);
-            sc.mig_waste = ceded % g.U[X];
+            sc.mig_m = (uint32_t)(avail / g.U[X]);
+            sc.mig_waste = avail % g.U[X];
             sc.newcap = sc.cap[Y] - (uint32_t)n;
             sc.fsm = AVMP_FSM_REBALANCING;
         }
@@ -135,8 +137,12 @@ __device__ void capacity_error(const Geom &g, Shared<NT> &sh, int X, unsigned lo
         sc.cap[Y] = newcap;
         sc.nfree[X] += m;
         sc.cap[X] += m;
-        sc.gap += sc.mig_waste;
-        sc.wasted += sc.mig_waste;
+        if (g.reclaim_gap) {
+            sc.gap = sc.mig_waste;          // the old gap went into the offer
+        } else {
+            sc.gap += sc.mig_waste;
+            sc.wasted += sc.mig_waste;
+        }
         sc.migrated += (unsigned long long)sc.mig_n * g.U[Y];
         sc.n_reb += 1;
         sc.last = counter;

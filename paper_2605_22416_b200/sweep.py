@@ -1,6 +1,6 @@
 """Sensitivity sweeps of the rebalancer on the synthetic workloads (paper Section 4.5):
 migration_batch_size B in {1 .. 256} (stage 1) and the threshold pairs (stage 2), plus the
-static partition, reporting the event-deterministic fields the paper tabulates -- OOM count,
+static partition and the default cell with the reclaim_gap variant of the waste rule, reporting the event-deterministic fields the paper tabulates -- OOM count,
 rebalance events, migrated MiB -- and, because this build really moves payload, relocated MiB
 and the device time spent relocating.
 
@@ -31,7 +31,7 @@ def run_cell(w: W.Workload, step_fn: Callable[[np.ndarray], np.ndarray], stats_f
     s = stats_fn()
     return {
         "B": w.migration_batch_size, "th_low": w.threshold_low_ppm / 1e6, "th_high": w.threshold_high_ppm / 1e6,
-        "dynamic": bool(w.migration_enabled), "steps": d.step, "ops": s["op_counter"], "n_oom": s["n_oom"],
+        "dynamic": bool(w.migration_enabled), "reclaim_gap": bool(w.reclaim_gap), "steps": d.step, "ops": s["op_counter"], "n_oom": s["n_oom"],
         "rebalances": s["n_rebalance"], "migrated_mib": s["migrated_bytes"] / W.MiB,
         "relocated_mib": s["relocated_bytes"] / W.MiB, "wasted_kib": s["wasted_bytes"] / 1024,
         "relocation_ms": s.get("relocation_ns_total", 0) / 1e6,
@@ -48,6 +48,7 @@ def cells(base: W.Workload, stage: str) -> List[W.Workload]:
         out += [base.with_(migration_batch_size=b) for b in B_VALUES]
     if stage in ("thresholds", "all"):
         out += [base.with_(threshold_low_ppm=lo, threshold_high_ppm=hi) for lo, hi in THRESHOLDS]
+    out.append(base.with_(reclaim_gap=True))
     return out
 
 
@@ -67,7 +68,7 @@ def gpu_cell(w: W.Workload, steps: int, device="cuda:0") -> Dict:
 
 
 def to_markdown(rows: List[Dict]) -> str:
-    cols = ("dynamic", "B", "th_low", "th_high", "n_oom", "rebalances", "migrated_mib", "relocated_mib",
+    cols = ("dynamic", "reclaim_gap", "B", "th_low", "th_high", "n_oom", "rebalances", "migrated_mib", "relocated_mib",
             "relocation_ms", "oom_retry_share", "migration_plan_share", "completed", "preempted", "cap_kv", "cap_ssm")
     lines = ["| " + " | ".join(cols) + " |", "|" + "---|" * len(cols)]
     for r in rows:

@@ -39,13 +39,14 @@ def test_library_is_loaded_from_the_tree(env):
     assert "libavmp.so" in maps
 
 
-def test_worked_example_on_gpu(env):
-    w = W.config("tiny")
+@pytest.mark.parametrize("golden,reclaim", [("worked_example.txt", False), ("worked_example_reclaim.txt", True)])
+def test_worked_example_on_gpu(env, golden, reclaim):
+    w = W.config("tiny", reclaim_gap=reclaim)
     g = env["GpuEngine"](w)
     kinds = {"ADMIT": 1, "EXTEND": 2, "FINISH": 3}
     cols = ("cap_kv", "free_kv", "cap_ssm", "free_ssm", "gap_bytes", "migrated_bytes", "wasted_bytes",
             "n_rebalance", "relocated_blocks", "n_oom", "n_capacity_error")
-    for line in (GOLDEN / "worked_example.txt").read_text().splitlines():
+    for line in (GOLDEN / golden).read_text().splitlines():
         if "|" not in line or line.startswith("#"):
             continue
         l, r = line.split("|")
@@ -56,6 +57,9 @@ def test_worked_example_on_gpu(env):
         assert int(st[0]) == exp[0], line
         assert [s[c] for c in cols] == exp[1:12], line
     pool, off, bad, aoff = g.translate(np.array([9, 8, 2, (1 << 31) | 2], np.uint32))
+    if reclaim:
+        assert bad == 0 and pool.tolist() == [0, 0, 0, 1] and off.tolist() == [576, 512, 0, 192]
+        return
     assert bad == 0 and pool.tolist() == [0, 0, 0, 1] and off.tolist() == [128, 512, 64, 192]
     # arena placement: KV grows up from 0, SSM slot j ends at pool_end - j * U
     assert aoff.tolist() == [128, 512, 64, 1024 - 3 * 96]
@@ -65,7 +69,7 @@ def test_worked_example_on_gpu(env):
 def test_random_op_strings_tiny(env, seed, batch):
     """Unscheduled ops (any order, repeated slots inside a batch, invalid ops): statuses,
     counters and every table equal the oracle's after each batch."""
-    w = W.config("tiny", migration_batch_size=1 + seed % 4)
+    w = W.config("tiny", migration_batch_size=1 + seed % 4, reclaim_gap=bool(seed % 2))
     g, o = _pair(env, w, max_requests=6, max_pages=8)
     ops = W.random_op_string(100 + seed, 3000, 6, 60)
     for i in range(0, len(ops), batch):
@@ -135,7 +139,7 @@ def test_random_shapes_and_policies(env, case):
     pool = int(rng.integers(10, 60)) * u
     w = W.Workload(f"rand{case}", shape, pool, float(rng.choice([0.0, 0.3, 0.5, 0.7, 1.0])), int(rng.integers(1, 9)),
                    8, 8, 6, "queue", 0, min_rebalance_interval_ops=int(rng.integers(1, 20)),
-                   threshold_high_ppm=int(rng.choice([100_000, 300_000, 500_000])))
+                   threshold_high_ppm=int(rng.choice([100_000, 300_000, 500_000])), reclaim_gap=case >= 7)
     g, o = _pair(env, w, with_store=True)
     for rnd in range(25):
         ops = W.random_op_string(case * 100 + rnd, int(rng.integers(1, 40)), 8, shape.page_tokens * 3, p_invalid=0.05)
@@ -321,6 +325,24 @@ def test_pr1_small_pool_relocations(env):
     assert s["relocated_blocks"] > 10 and s["n_rebalance"] > 5
 
 
+@pytest.mark.parametrize("name,steps,over", [
+    ("pr1", 1200, dict(pool_bytes=24 * W.MiB, concurrency=12, min_rebalance_interval_ops=50,
+                       migration_batch_size=6, n_requests=300)),
+    ("mixed_long", 300, dict(migration_batch_size=4)),
+])
+def test_reclaim_gap_variant(env, name, steps, over):
+    """The variant of the waste rule that offers the gap between the pools again: same closed loop,
+    same comparisons; capacities must differ from the paper's rule on the same trace prefix."""
+    w = W.config(name, reclaim_gap=True, **over)
+    small = name == "pr1"
+    s, seen, d = _closed_loop_parity(env, w, steps, with_store=small, kv_layers=[1], ssm_layers=[3],
+                                     table_every=1 if small else 64, gather_every=5 if small else 97,
+                                     max_migration_checks=12)
+    assert s["n_rebalance"] > 3 and s["wasted_bytes"] == 0
+    u = (s["unit_bytes_kv"], s["unit_bytes_ssm"])
+    assert s["gap_bytes"] < max(u)          # never a whole recipient unit left lying
+
+
 def test_multi_layer_gathers(env):
     """avmp_gather_kv_layers / avmp_gather_ssm_layers: one launch for a range of layers gives,
     layer by layer, the oracle's single-layer gathers (and the payload function's bytes)."""
@@ -472,7 +494,7 @@ def test_sensitivity_sweep_cells_match_the_oracle(env):
     # static partition event for event (the paper's B = 1 row equals its static total too)
     assert all(b1[k] == static[k] for k in ("n_oom", "rebalances", "completed", "ops", "cap_kv", "cap_ssm"))
     assert any(r["rebalances"] > 0 and r["relocated_mib"] > 0 for r in rows_o)
-    th = [r for r in rows_o if r["dynamic"] and r["B"] == base.migration_batch_size]
+    th = [r for r in rows_o if r["dynamic"] and r["B"] == base.migration_batch_size and not r["reclaim_gap"]]
     ref = {k: v for k, v in th[0].items() if k not in ("th_low",)}
     same_high = [r for r in th if r["th_high"] == th[0]["th_high"]]
     assert len(same_high) >= 3
@@ -483,6 +505,7 @@ def test_sensitivity_sweep_cells_match_the_oracle(env):
 @pytest.mark.parametrize("name,steps,over", [
     ("pr1", 900, dict(pool_bytes=40 * W.MiB, min_rebalance_interval_ops=100)),       # OOMs, pre-emptions
     ("pr1", 400, dict(pool_bytes=8 * W.MiB, migration_enabled=False, n_requests=300)),  # unservable drops
+    ("pr1", 500, dict(pool_bytes=40 * W.MiB, min_rebalance_interval_ops=100, reclaim_gap=True)),
     ("short_uniform", 500, {}),
     ("mixed_long", 400, dict(migration_batch_size=64)),
     ("scale", 60, {}),
