@@ -65,11 +65,22 @@ def _mix64(x: np.ndarray) -> np.ndarray:
     return x
 
 
+_M64 = 0xFFFFFFFFFFFFFFFF
+
+
+def _mix64_int(x: int) -> int:
+    """The same function on one Python integer."""
+    x ^= x >> 30
+    x = (x * 0xBF58476D1CE4E5B9) & _M64
+    x ^= x >> 27
+    x = (x * 0x94D049BB133111EB) & _M64
+    return x ^ (x >> 31)
+
+
 def _key(seed: int, stream: int) -> np.uint64:
-    with np.errstate(over="ignore"):
-        a = _mix64(np.array([seed & 0xFFFFFFFFFFFFFFFF], dtype=np.uint64))[0]
-        b = _mix64(np.array([(stream + 0x1234567) & 0xFFFFFFFFFFFFFFFF], dtype=np.uint64) * _GOLDEN)[0]
-        return _mix64(np.array([a ^ b], dtype=np.uint64))[0]
+    a = _mix64_int(seed & _M64)
+    b = _mix64_int((((stream + 0x1234567) & _M64) * 0x9E3779B97F4A7C15) & _M64)
+    return np.uint64(_mix64_int(a ^ b))
 
 
 def rand_u64(seed: int, stream: int, n: int, start: int = 0) -> np.ndarray:
@@ -133,6 +144,24 @@ def payload_bytes(seed: int, uid: int, epoch: int, layer: int, part: int,
         w = _mix64(k + (idx + np.uint64(1)) * _GOLDEN)
     b = w.astype("<u8").view(np.uint8)[b0 - w0 * 8: b1 - w0 * 8]
     return b.reshape(n_rows, row_bytes)
+
+
+def payload_single_rows(seed: int, uids, epochs, layer: int, part: int, rows, row_bytes: int) -> np.ndarray:
+    """uint8[n, row_bytes]: row rows[i] of the stream of (uids[i], epochs[i]) -- the same bytes as
+    one payload_bytes call per item, computed in one pass when rows are whole 8-byte words."""
+    n = len(uids)
+    if n == 0:
+        return np.zeros((0, row_bytes), np.uint8)
+    if row_bytes % 8:
+        return np.concatenate([payload_bytes(seed, int(u), int(e), layer, part, int(r), 1, row_bytes)
+                               for u, e, r in zip(uids, epochs, rows)])
+    wpr = row_bytes // 8
+    keys = np.array([_key(seed ^ 0x5EED, (int(u) * 64 + int(e)) * 4096 + layer * 4 + part)
+                     for u, e in zip(uids, epochs)], dtype=np.uint64)
+    with np.errstate(over="ignore"):
+        idx = (np.asarray(rows, dtype=np.uint64) * np.uint64(wpr))[:, None] + np.arange(wpr, dtype=np.uint64)[None, :]
+        w = _mix64(keys[:, None] + (idx + np.uint64(1)) * _GOLDEN)
+    return w.astype("<u8").view(np.uint8).reshape(n, row_bytes)
 
 
 # ----------------------------------------------------------------------------

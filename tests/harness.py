@@ -27,18 +27,29 @@ class PayloadHarness:
         m = self.w.model
         slots = np.array([x.slot for x in writes], np.uint32)
         starts = np.array([x.start for x in writes], np.uint32)
+        # single-token writes (the EXTENDs) first, in one pass; the scatter order is free
+        one = [i for i, x in enumerate(writes) if x.end - x.start == 1]
+        many = [i for i, x in enumerate(writes) if x.end - x.start != 1]
+        order = one + many
+        slots, starts = slots[order], starts[order]
+        u1 = [writes[i].uid for i in one]
+        r1 = [writes[i].start for i in one]
         for layer in self.kv_layers:
-            ks = [W.payload_bytes(self.seed, x.uid, 0, layer, W.PAYLOAD_K, x.start, x.end - x.start, m.kv_row_bytes) for x in writes]
-            vs = [W.payload_bytes(self.seed, x.uid, 0, layer, W.PAYLOAD_V, x.start, x.end - x.start, m.kv_row_bytes) for x in writes]
-            in_k, in_v = np.concatenate(ks), np.concatenate(vs)
+            parts = []
+            for part in (W.PAYLOAD_K, W.PAYLOAD_V):
+                rows = [W.payload_single_rows(self.seed, u1, [0] * len(u1), layer, part, r1, m.kv_row_bytes)]
+                rows += [W.payload_bytes(self.seed, writes[i].uid, 0, layer, part, writes[i].start,
+                                         writes[i].end - writes[i].start, m.kv_row_bytes) for i in many]
+                parts.append(np.concatenate(rows))
             for e in self.engines:
-                assert e.scatter_kv(layer, slots, starts, in_k, in_v) == 0
+                assert e.scatter_kv(layer, slots, starts, parts[0], parts[1]) == 0
         adm = [x for x in writes if x.is_admit]
         if adm:
             aslots = np.array([x.slot for x in adm], np.uint32)
             for layer in self.ssm_layers:
-                st = np.concatenate([W.payload_bytes(self.seed, x.uid, x.epoch, layer, W.PAYLOAD_STATE, 0, 1, m.state_bytes) for x in adm])
-                cv = np.concatenate([W.payload_bytes(self.seed, x.uid, x.epoch, layer, W.PAYLOAD_CONV, 0, 1, m.conv_bytes) for x in adm])
+                au, ae, z = [x.uid for x in adm], [x.epoch for x in adm], [0] * len(adm)
+                st = W.payload_single_rows(self.seed, au, ae, layer, W.PAYLOAD_STATE, z, m.state_bytes)
+                cv = W.payload_single_rows(self.seed, au, ae, layer, W.PAYLOAD_CONV, z, m.conv_bytes)
                 for e in self.engines:
                     assert e.scatter_ssm(layer, aslots, st, cv) == 0
 
@@ -53,10 +64,9 @@ class PayloadHarness:
 
     def expected_ssm(self, layer: int, uids, epochs):
         m = self.w.model
-        st = [W.payload_bytes(self.seed, int(u), int(e), layer, W.PAYLOAD_STATE, 0, 1, m.state_bytes) for u, e in zip(uids, epochs)]
-        cv = [W.payload_bytes(self.seed, int(u), int(e), layer, W.PAYLOAD_CONV, 0, 1, m.conv_bytes) for u, e in zip(uids, epochs)]
-        return (np.concatenate(st or [np.zeros((0, m.state_bytes), np.uint8)]),
-                np.concatenate(cv or [np.zeros((0, m.conv_bytes), np.uint8)]))
+        z = [0] * len(uids)
+        return (W.payload_single_rows(self.seed, uids, epochs, layer, W.PAYLOAD_STATE, z, m.state_bytes),
+                W.payload_single_rows(self.seed, uids, epochs, layer, W.PAYLOAD_CONV, z, m.conv_bytes))
 
     def check_gathers(self, d: W.ClosedLoopDriver, kv_layer: int, ssm_layer: int, engines=None) -> int:
         """Gather the whole running batch from every engine and compare with the payload
