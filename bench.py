@@ -425,9 +425,14 @@ def device_closed_loop(dev, workload: str, steps: int = 3000) -> dict:
     out = {"workload": workload, "steps": steps}
     for label, enabled in (("dynamic", True), ("static", False)):
         w = W.config(workload, migration_enabled=enabled)
-        reqs = W.make_requests(w, min(w.n_requests, 200_000))
         ctx = B.Context.from_workload(w, device=dev)
-        dd = B.DeviceDriver(ctx, reqs.prompt, reqs.output, w.concurrency)
+        if w.kind == "sessions":
+            ses = W.make_sessions(w)
+            dd = B.SessionDriver(ctx, ses.arrival_step, ses.n_turns, ses.turn_prompt, ses.turn_output,
+                                 ses.turn_think, w.concurrency)
+        else:
+            reqs = W.make_requests(w, min(w.n_requests, 200_000))
+            dd = B.DeviceDriver(ctx, reqs.prompt, reqs.output, w.concurrency)
         sid = torch.cuda.current_stream().cuda_stream
         torch.cuda.synchronize(dev)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

@@ -329,6 +329,46 @@ AVMP_API int avmp_driver_get_stats(avmp_driver *drv, avmp_driver_stats *h_out, v
 AVMP_API int avmp_driver_export(avmp_driver *drv, uint32_t *h_state, uint32_t *h_uid, uint32_t *h_len,
                                 uint32_t *h_remaining, void *stream);
 
+/* ---- the same loop for multi-turn sessions (the agentic-burst workload; the paper gives that
+ * workload one sentence in Section 4.1 and no scheduler, so the policy is this library's) ----
+ * Sessions arrive at d_arrival_step[i] (ascending); turn t of session i appends d_turn_prompt[i *
+ * max_turns + t] prompt tokens and decodes d_turn_output[...] tokens; between turns the request
+ * parks (FINISH with KEEP_KV) for d_turn_think[i * max_turns + t] steps and then resumes on its own
+ * slot (ADMIT with RESUME); after turn d_n_turns[i] - 1 it finishes for good.  Each step admits, in
+ * this order, re-queued entries, parked sessions whose think time is over (by ready step, then by
+ * parking order) and newly arrived sessions, within the concurrency and the slow-start window;
+ * a step that saw an OOM or ran out of free slots evicts the longest-parked chain (that session re-enters with its whole
+ * context as the prompt), a step without any success pre-empts the most recently admitted
+ * request, an admit that fails with nothing running and nothing parked is dropped.
+ * All five arrays are device arrays of uint32 owned by the caller and must outlive the driver;
+ * concurrency <= 1024.  The workspace (avmp_session_driver_workspace_bytes, 256-byte aligned) is
+ * the caller's.  Each step is a few stream-ordered launches with no host round trip. */
+typedef struct avmp_session_driver avmp_session_driver;
+typedef struct {
+    uint64_t steps, completed, dropped, preempted, evicted, n_oom_admit, n_oom_extend;
+    uint64_t arrived;         /* sessions whose arrival step has passed */
+    uint64_t arrival_queue;   /* of those, still waiting for their first admission */
+    uint64_t requeued;        /* entries at the queue head (failed admits, pre-empted, found no slot) */
+    uint64_t waiting;         /* parked or evicted sessions waiting for their ready step */
+    uint64_t window, last_batch_ops;
+    uint64_t forced_slot;     /* slot the next step will pre-empt or evict, ~0 if none */
+} avmp_session_stats;
+AVMP_API size_t avmp_session_driver_workspace_bytes(uint32_t max_requests, uint32_t n_sessions);
+AVMP_API int avmp_session_driver_create(avmp_session_driver **out, avmp_ctx *ctx, const uint32_t *d_arrival_step,
+                                        const uint32_t *d_n_turns, const uint32_t *d_turn_prompt,
+                                        const uint32_t *d_turn_output, const uint32_t *d_turn_think,
+                                        uint32_t n_sessions, uint32_t max_turns, uint32_t concurrency,
+                                        void *d_workspace, size_t workspace_bytes, void *stream);
+AVMP_API int avmp_session_driver_destroy(avmp_session_driver *drv);
+AVMP_API int avmp_session_driver_step(avmp_session_driver *drv, void *stream);
+/* Both synchronise the stream.  Export copies the per-slot arrays (state 0 free / 1 running / 2
+ * parked, session index, tokens held, decode tokens left, turn), max_requests entries each, and the
+ * session indices in the re-queued and the waiting queue, in order (room for n_sessions each). */
+AVMP_API int avmp_session_driver_get_stats(avmp_session_driver *drv, avmp_session_stats *h_out, void *stream);
+AVMP_API int avmp_session_driver_export(avmp_session_driver *drv, uint32_t *h_state, uint32_t *h_uid, uint32_t *h_len,
+                                        uint32_t *h_remaining, uint32_t *h_turn, uint32_t *h_requeued,
+                                        uint32_t *h_waiting, void *stream);
+
 /* How many kernels this context has launched so far (host counter). */
 AVMP_API uint64_t avmp_launch_count(const avmp_ctx *ctx);
 

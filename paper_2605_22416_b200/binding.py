@@ -63,6 +63,14 @@ class avmp_driver_stats(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in DRIVER_STAT_FIELDS]
 
 
+SESSION_STAT_FIELDS = ("steps", "completed", "dropped", "preempted", "evicted", "n_oom_admit", "n_oom_extend",
+                       "arrived", "arrival_queue", "requeued", "waiting", "window", "last_batch_ops", "forced_slot")
+
+
+class avmp_session_stats(C.Structure):
+    _fields_ = [(n, C.c_uint64) for n in SESSION_STAT_FIELDS]
+
+
 _u32p = C.POINTER(C.c_uint32)
 
 
@@ -93,6 +101,13 @@ def _load():
         "avmp_driver_step": (C.c_int, [vp, vp]),
         "avmp_driver_get_stats": (C.c_int, [vp, C.POINTER(avmp_driver_stats), vp]),
         "avmp_driver_export": (C.c_int, [vp, vp, vp, vp, vp, vp]),
+        "avmp_session_driver_workspace_bytes": (C.c_size_t, [C.c_uint32, C.c_uint32]),
+        "avmp_session_driver_create": (C.c_int, [C.POINTER(vp), vp, vp, vp, vp, vp, vp, C.c_uint32, C.c_uint32,
+                                                 C.c_uint32, vp, C.c_size_t, vp]),
+        "avmp_session_driver_destroy": (C.c_int, [vp]),
+        "avmp_session_driver_step": (C.c_int, [vp, vp]),
+        "avmp_session_driver_get_stats": (C.c_int, [vp, C.POINTER(avmp_session_stats), vp]),
+        "avmp_session_driver_export": (C.c_int, [vp, vp, vp, vp, vp, vp, vp, vp, vp]),
         "avmp_translate": (C.c_int, [vp, vp, C.c_uint32, vp, vp, vp, vp]),
         "avmp_gather_kv": (C.c_int, [vp, C.c_uint32, vp, C.c_uint32, vp, vp, C.c_uint64, vp, vp]),
         "avmp_gather_kv_static": (C.c_int, [vp, C.c_uint32, vp, C.c_uint32, vp, vp, C.c_uint64, vp, vp]),
@@ -223,6 +238,44 @@ def avmp_driver_export(drv, max_requests: int, stream=None) -> dict:
     a = {k: np.zeros(max_requests, np.uint32) for k in ("state", "uid", "len", "remaining")}
     _check(lib.avmp_driver_export(drv, _ptr(a["state"]), _ptr(a["uid"]), _ptr(a["len"]), _ptr(a["remaining"]),
                                   _stream(stream)), "avmp_driver_export")
+    return a
+
+
+def avmp_session_driver_workspace_bytes(max_requests: int, n_sessions: int) -> int:
+    return lib.avmp_session_driver_workspace_bytes(max_requests, n_sessions)
+
+
+def avmp_session_driver_create(ctx, d_arrival_step, d_n_turns, d_turn_prompt, d_turn_output, d_turn_think,
+                               n_sessions, max_turns, concurrency, d_workspace, workspace_bytes, stream=None) -> int:
+    h = C.c_void_p()
+    _check(lib.avmp_session_driver_create(C.byref(h), ctx, _ptr(d_arrival_step), _ptr(d_n_turns), _ptr(d_turn_prompt),
+                                          _ptr(d_turn_output), _ptr(d_turn_think), n_sessions, max_turns, concurrency,
+                                          _ptr(d_workspace), workspace_bytes, _stream(stream)),
+           "avmp_session_driver_create")
+    return h.value
+
+
+def avmp_session_driver_destroy(drv):
+    _check(lib.avmp_session_driver_destroy(drv), "avmp_session_driver_destroy")
+
+
+def avmp_session_driver_step(drv, stream=None):
+    _check(lib.avmp_session_driver_step(drv, _stream(stream)), "avmp_session_driver_step")
+
+
+def avmp_session_driver_get_stats(drv, stream=None) -> dict:
+    s = avmp_session_stats()
+    _check(lib.avmp_session_driver_get_stats(drv, C.byref(s), _stream(stream)), "avmp_session_driver_get_stats")
+    return {k: int(getattr(s, k)) for k in SESSION_STAT_FIELDS}
+
+
+def avmp_session_driver_export(drv, max_requests: int, n_sessions: int, stream=None) -> dict:
+    a = {k: np.zeros(max_requests, np.uint32) for k in ("state", "uid", "len", "remaining", "turn")}
+    a["requeued"] = np.zeros(n_sessions, np.uint32)
+    a["waiting"] = np.zeros(n_sessions, np.uint32)
+    _check(lib.avmp_session_driver_export(drv, _ptr(a["state"]), _ptr(a["uid"]), _ptr(a["len"]), _ptr(a["remaining"]),
+                                          _ptr(a["turn"]), _ptr(a["requeued"]), _ptr(a["waiting"]), _stream(stream)),
+           "avmp_session_driver_export")
     return a
 
 
@@ -501,6 +554,56 @@ class DeviceDriver:
             avmp_driver_destroy(self.handle)
             self.handle = None
             self.workspace = self.d_prompt = self.d_output = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class SessionDriver:
+    """Owner of the on-device closed loop for multi-turn sessions: uploads the session arrays
+    (arrival step, turns, per-turn prompt / output / think time), allocates the workspace, forwards
+    to the avmp_session_driver_* entry points."""
+
+    def __init__(self, ctx: Context, arrival_step, n_turns, turn_prompt, turn_output, turn_think, concurrency: int):
+        self.ctx = ctx
+        dev = ctx.device
+        self.n_sessions = len(arrival_step)
+        self.max_turns = int(np.asarray(turn_prompt).shape[1])
+
+        def up(a):
+            return torch.from_numpy(np.ascontiguousarray(a, dtype=np.uint32).view(np.int32).reshape(-1)).to(dev)
+
+        self.arrays = [up(a) for a in (arrival_step, n_turns, turn_prompt, turn_output, turn_think)]
+        ws = avmp_session_driver_workspace_bytes(ctx.opt.max_requests, self.n_sessions)
+        if ws == 0:
+            raise AvmpError("avmp_session_driver_workspace_bytes rejected the sizes")
+        with torch.cuda.device(dev):
+            self.workspace = torch.empty(ws, dtype=torch.uint8, device=dev)
+            self.handle = avmp_session_driver_create(ctx.handle, *self.arrays, self.n_sessions, self.max_turns,
+                                                     concurrency, self.workspace, ws)
+
+    def step(self, stream=None):
+        avmp_session_driver_step(self.handle, stream)
+
+    def stats(self, stream=None) -> dict:
+        return avmp_session_driver_get_stats(self.handle, stream)
+
+    def export(self, stream=None) -> dict:
+        s = self.stats(stream)
+        a = avmp_session_driver_export(self.handle, self.ctx.opt.max_requests, self.n_sessions, stream)
+        a["requeued"] = a["requeued"][:s["requeued"]]
+        a["waiting"] = a["waiting"][:s["waiting"]]
+        return a
+
+    def close(self):
+        if getattr(self, "handle", None):
+            torch.cuda.synchronize(self.ctx.device)
+            avmp_session_driver_destroy(self.handle)
+            self.handle = None
+            self.workspace = self.arrays = None
 
     def __del__(self):
         try:

@@ -348,9 +348,9 @@ class ClosedLoopDriver:
     most recently admitted running request (plain FINISH, re-queued at the head with
     its whole context as the prompt).  An admit that fails with nothing running is
     dropped as unservable.  Multi-turn sessions park between turns (FINISH with
-    KEEP_KV) and resume after their think time; a step that ran out of memory evicts
-    the longest-parked session's chain (plain FINISH; it re-enters as a fresh admit
-    with its whole context as the prompt).
+    KEEP_KV) and resume after their think time; a step that ran out of memory, or in
+    which an admission found no free slot, evicts the longest-parked session's chain
+    (plain FINISH; it re-enters as a fresh admit with its whole context as the prompt).
     """
 
     def __init__(self, w: Workload, requests: Optional[RequestList] = None,
@@ -373,6 +373,7 @@ class ClosedLoopDriver:
         self.parked: dict = {}                  # slot -> (park_seq, entry)
         self.window = w.concurrency
         self._forced: dict = {}                 # slot -> "preempt" | "drop" | "evict"
+        self._starved = False                   # the last batch left an entry without a slot
         self.completed = self.dropped = self.preempted = self.evicted = 0
         self.n_oom_admit = self.n_oom_extend = 0
         self.writes: List[TokenWrite] = []
@@ -443,6 +444,7 @@ class ClosedLoopDriver:
         budget = min(self.w.concurrency - len(ext), self.window)
         free_slots = np.flatnonzero(self.state == _FREE)
         n_free_used = 0
+        self._starved = False
         admits: List[Tuple[_Entry, int]] = []
         while budget > 0:
             e = self._pop_entry()
@@ -455,6 +457,7 @@ class ClosedLoopDriver:
                 n_free_used += 1
             else:
                 self.front.appendleft(e)
+                self._starved = True
                 break
             admits.append((e, slot))
             budget -= 1
@@ -569,7 +572,7 @@ class ClosedLoopDriver:
             self.dropped += 1
         for e in reversed(failed):
             self.front.appendleft(e)
-        if oom_seen and self.parked:
+        if (oom_seen or self._starved) and self.parked:
             slot = min(self.parked, key=lambda s: self.parked[s][0])
             self._forced[slot] = "evict"
         elif not progress and n_running > 0 and len(status) > 0:

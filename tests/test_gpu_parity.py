@@ -546,6 +546,55 @@ def test_device_closed_loop_matches_host_loop(env, name, steps, over):
     dd.close()
 
 
+@pytest.mark.parametrize("steps,over", [
+    (1500, {}),
+    (1200, dict(pool_bytes=3 * W.GiB)),                                  # tight: evictions, failed resumes
+    (900, dict(pool_bytes=2 * W.GiB, concurrency=64, split=0.3)),         # pre-emptions, no free slot
+    (700, dict(pool_bytes=3 * W.GiB, max_requests=96, concurrency=96)),   # slots run out before memory
+    (600, dict(pool_bytes=3 * W.GiB, reclaim_gap=True, migration_batch_size=32)),
+    (800, dict(max_requests=24, concurrency=24)),                         # parked sessions hold every slot
+])
+def test_device_session_loop_matches_host_loop(env, steps, over):
+    """The on-device scheduler for multi-turn sessions (arrivals, parking with KEEP_KV, resume after the
+    think time, eviction of the longest-parked chain, pre-emption, drops) against the host-side batch
+    builder running on the oracle: allocator tables and counters, every slot, both queues in order and
+    every scheduler counter, compared every 100 steps."""
+    from paper_2605_22416_b200 import binding as B
+    w = W.config("agentic_burst", **over)
+    ses = W.make_sessions(w)
+    g = env["GpuEngine"](w)
+    sd = B.SessionDriver(g.ctx, ses.arrival_step, ses.n_turns, ses.turn_prompt, ses.turn_output, ses.turn_think,
+                         w.concurrency)
+    o = env["Oracle"].from_workload(w)
+    d = W.ClosedLoopDriver(w, sessions=ses)
+    done = 0
+    while done < steps:
+        n = min(100, steps - done)
+        for _ in range(n):
+            sd.step()
+            d.feed(o.step(d.next_batch()))
+        done += n
+        what = f"session loop at step {done}"
+        ds, ex = sd.stats(), sd.export()
+        for k in ("completed", "dropped", "preempted", "evicted", "n_oom_admit", "n_oom_extend", "window"):
+            assert ds[k] == getattr(d, k), (what, k, ds[k], getattr(d, k))
+        assert ds["steps"] == done and ds["arrived"] == d._next and ds["arrival_queue"] == len(d.back), what
+        assert ex["requeued"].tolist() == [e.uid for e in d.front], what
+        assert ex["waiting"].tolist() == [e.uid for _, _, e in d.resume_q], what
+        forced = list(d._forced)
+        assert ds["forced_slot"] == (forced[0] if forced else 2**64 - 1), what
+        assert np.array_equal(ex["state"], d.state.astype(np.uint32)), what
+        held = d.state != 0
+        for k, a in (("uid", d.uid), ("len", d.len), ("turn", d.turn)):
+            assert np.array_equal(ex[k][held], a[held].astype(np.uint32)), (what, k)
+        run = d.state == 1
+        assert np.array_equal(ex["remaining"][run], d.remaining[run].astype(np.uint32)), what
+        env["same"](g, o, w, what)
+    assert g.stats()["error_code"] == 0
+    assert d.completed > 0 and (d.evicted > 0 or (d.state == 2).any())
+    sd.close()
+
+
 def test_device_loop_replayed_from_a_cuda_graph(env):
     """Fifty engine steps of the on-device loop captured once in a CUDA graph and replayed ten
     times: same final state as five hundred steps of the host loop on the oracle."""
