@@ -138,12 +138,32 @@ def payload_bytes(seed: int, uid: int, epoch: int, layer: int, part: int,
     b0 = row_start * row_bytes
     b1 = (row_start + n_rows) * row_bytes
     w0, w1 = b0 // 8, -(-b1 // 8)
-    with np.errstate(over="ignore"):
-        k = _key(seed ^ 0x5EED, (uid * 64 + epoch) * 4096 + layer * 4 + part)
-        idx = np.arange(w0, w1, dtype=np.uint64)
-        w = _mix64(k + (idx + np.uint64(1)) * _GOLDEN)
-    b = w.astype("<u8").view(np.uint8)[b0 - w0 * 8: b1 - w0 * 8]
+    w = _stream_words(_key(seed ^ 0x5EED, (uid * 64 + epoch) * 4096 + layer * 4 + part), w0, w1)
+    b = w.astype("<u8", copy=False).view(np.uint8)[b0 - w0 * 8: b1 - w0 * 8]
     return b.reshape(n_rows, row_bytes)
+
+
+def _stream_words(k: np.uint64, w0: int, w1: int, chunk: int = 1 << 16) -> np.ndarray:
+    """Words [w0, w1) of the stream with key k: mix64(k + (i + 1) * golden).  Generated in
+    cache-sized pieces with in-place arithmetic; long streams would otherwise be bound by the
+    page faults of their temporaries."""
+    out = np.empty(w1 - w0, np.uint64)
+    with np.errstate(over="ignore"):
+        for s in range(w0, w1, chunk):
+            e = min(s + chunk, w1)
+            x = np.arange(s + 1, e + 1, dtype=np.uint64)
+            x *= _GOLDEN
+            x += k
+            t = x >> np.uint64(30)
+            x ^= t
+            x *= np.uint64(0xBF58476D1CE4E5B9)
+            np.right_shift(x, np.uint64(27), out=t)
+            x ^= t
+            x *= np.uint64(0x94D049BB133111EB)
+            np.right_shift(x, np.uint64(31), out=t)
+            x ^= t
+            out[s - w0:e - w0] = x
+    return out
 
 
 def payload_single_rows(seed: int, uids, epochs, layer: int, part: int, rows, row_bytes: int) -> np.ndarray:
