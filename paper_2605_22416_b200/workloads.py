@@ -172,9 +172,11 @@ def payload_single_rows(seed: int, uids, epochs, layer: int, part: int, rows, ro
     n = len(uids)
     if n == 0:
         return np.zeros((0, row_bytes), np.uint8)
-    if row_bytes % 8:
-        return np.concatenate([payload_bytes(seed, int(u), int(e), layer, part, int(r), 1, row_bytes)
-                               for u, e, r in zip(uids, epochs, rows)])
+    if row_bytes % 8 or row_bytes > 8192:      # long rows: one cache-sized stream at a time
+        out = np.empty((n, row_bytes), np.uint8)
+        for i, (u, e, r) in enumerate(zip(uids, epochs, rows)):
+            out[i] = payload_bytes(seed, int(u), int(e), layer, part, int(r), 1, row_bytes)[0]
+        return out
     wpr = row_bytes // 8
     keys = np.array([_key(seed ^ 0x5EED, (int(u) * 64 + int(e)) * 4096 + layer * 4 + part)
                      for u, e in zip(uids, epochs)], dtype=np.uint64)
