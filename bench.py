@@ -347,7 +347,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
                       "note": "avmp_step + avmp_translate, CUDA events around the two calls, rank 0's timing"},
         "gather_kv": {"gbs": kv_launch_bytes / (kv_avg_ms * 1e-3) / 1e9, "avg_launch_ms": kv_avg_ms,
                       "frac_of_peak": kv_launch_bytes / (kv_avg_ms * 1e-3) / 1e9 / peak,
-                      "note": "avmp_gather_kv_layers: plan kernel + one copy launch for all attention layers"},
+                      "note": "avmp_gather_kv_layers: one copy launch for all attention layers (the request-list plan is computed inside it)"},
         "per_layer_launches": {"gather_ssm_gbs": pl_ssm, "gather_ssm_frac_of_peak": pl_ssm / peak,
                                "gather_ssm_avg_launch_ms": float(np.mean(per_l["ssm"])),
                                "gather_kv_gbs": pl_kv, "gather_kv_frac_of_peak": pl_kv / peak,

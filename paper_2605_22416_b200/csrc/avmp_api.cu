@@ -270,7 +270,7 @@ int avmp_gather_kv(avmp_ctx *c, uint32_t layer, const uint32_t *d_reqs, uint32_t
     if (!c || layer >= c->spec.n_attn_layers || n > c->opt.max_requests || !d_cu) return AVMP_EINVAL;
     if (n && (!d_reqs || !d_out_k || !d_out_v)) return AVMP_EINVAL;
     if (((uintptr_t)d_out_k | (uintptr_t)d_out_v) & 15) return AVMP_EINVAL;
-    c->launches += 2;
+    c->launches += n > kLocalPlanMax ? 2 : 1;      // a separate plan launch only for long lists
     return cu(launch_kv(c->g, false, layer, 1, d_reqs, nullptr, n, d_out_k, d_out_v, 0, cap_tokens, d_cu, L(c, stream)));
 }
 
@@ -280,7 +280,7 @@ int avmp_scatter_kv(avmp_ctx *c, uint32_t layer, const uint32_t *d_reqs, const u
     if (!c || layer >= c->spec.n_attn_layers || n > c->opt.max_requests) return AVMP_EINVAL;
     if (n == 0) return AVMP_OK;
     if (!d_reqs || !d_in_k || !d_in_v || (((uintptr_t)d_in_k | (uintptr_t)d_in_v) & 15)) return AVMP_EINVAL;
-    c->launches += 2;
+    c->launches += n > kLocalPlanMax ? 2 : 1;      // a separate plan launch only for long lists
     return cu(launch_kv(c->g, true, layer, 1, d_reqs, d_tok_start, n, const_cast<void *>(d_in_k),
                         const_cast<void *>(d_in_v), 0, ~0ull, nullptr, L(c, stream)));
 }
@@ -315,7 +315,7 @@ int avmp_gather_kv_layers(avmp_ctx *c, uint32_t first_layer, uint32_t n_layers, 
     if (n && (!d_reqs || !d_out_k || !d_out_v)) return AVMP_EINVAL;
     if (((uintptr_t)d_out_k | (uintptr_t)d_out_v | layer_stride_bytes) & 15) return AVMP_EINVAL;
     if (n_layers > 1 && layer_stride_bytes < cap_tokens * c->lay.kv_row_bytes) return AVMP_EINVAL;
-    c->launches += 2;
+    c->launches += n > kLocalPlanMax ? 2 : 1;      // a separate plan launch only for long lists
     return cu(launch_kv(c->g, false, first_layer, n_layers, d_reqs, nullptr, n, d_out_k, d_out_v, layer_stride_bytes,
                         cap_tokens, d_cu, L(c, stream)));
 }
@@ -342,7 +342,7 @@ int avmp_scatter_kv_layers(avmp_ctx *c, uint32_t first_layer, uint32_t n_layers,
     if (!c || n_layers == 0 || (uint64_t)first_layer + n_layers > c->spec.n_attn_layers || n > c->opt.max_requests) return AVMP_EINVAL;
     if (n == 0) return AVMP_OK;
     if (!d_reqs || !d_in_k || !d_in_v || (((uintptr_t)d_in_k | (uintptr_t)d_in_v | layer_stride_bytes) & 15)) return AVMP_EINVAL;
-    c->launches += 2;
+    c->launches += n > kLocalPlanMax ? 2 : 1;      // a separate plan launch only for long lists
     return cu(launch_kv(c->g, true, first_layer, n_layers, d_reqs, d_tok_start, n, const_cast<void *>(d_in_k),
                         const_cast<void *>(d_in_v), layer_stride_bytes, ~0ull, nullptr, L(c, stream)));
 }

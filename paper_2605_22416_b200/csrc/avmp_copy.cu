@@ -67,6 +67,7 @@ struct Piece {
 template <bool SCATTER>
 struct SsmPieces {
     static constexpr bool kTimed = false;
+    static constexpr bool kPlans = false;
     uint32_t layer0, n_layers, n, ps, per;
     const uint32_t *reqs;
     uint8_t *buf_state, *buf_conv;
@@ -107,6 +108,7 @@ struct SsmPieces {
 // a7: chunks of the units moved by the last migration.
 struct RelocPieces {
     static constexpr bool kTimed = true;     // the copy stamps the device clock: migration time is a metric
+    static constexpr bool kPlans = false;
     __device__ unsigned long long total(const Geom &g) const
     {
         const unsigned long long U = g.U[g.st->reloc_pool];
@@ -125,26 +127,77 @@ struct RelocPieces {
     }
 };
 
-// a11: slices of the pages of a KV chain <-> rows of the ragged batch buffers.  The plan
-// kernel has written, per request k, the first row (g_cu_rows) and the first piece
-// (g_cu_items); a request spanning P pages owns P * subs pieces, `subs` = slices per page
-// (K slices, then V slices).
+// a11: slices of the pages of a KV chain <-> rows of the ragged batch buffers.  A plan gives,
+// per request k, the first row (cu_rows) and the first piece (cu_items); a request spanning P
+// pages owns P * subs pieces, `subs` = slices per page (K slices, then V slices).  For request
+// lists of up to kLocalPlanMax entries every CTA of the copy computes the plan itself into its
+// shared memory (a few hundred table reads and a block scan: cheaper than a separate launch and
+// its dependency, and calls on different streams share no scratch); longer lists use the plan
+// kernel and the context's global scratch.
+// One request's rows and pieces for a KV gather / scatter (errors recorded by the caller's choice).
+__device__ __forceinline__ void kv_plan_entry(const Geom &g, const uint32_t *reqs, const uint32_t *tok_start,
+                                              uint32_t k, uint32_t subs, bool report, uint32_t &rows, uint32_t &items)
+{
+    rows = 0; items = 0;
+    const uint32_t r = reqs[k];
+    const uint32_t st = r < g.R ? g.r_state[r] : AVMP_REQ_EMPTY;
+    const uint32_t t0 = tok_start ? tok_start[k] : 0u;
+    if (st == AVMP_REQ_EMPTY) { if (report) record_error(g.st, AVMP_DEV_BAD_REQUEST); }
+    else {
+        const uint32_t len = g.r_len[r];
+        if (t0 > len) { if (report) record_error(g.st, AVMP_DEV_BAD_REQUEST); }
+        else rows = len - t0;
+    }
+    if (rows) items = ((t0 + rows - 1u) / g.T - t0 / g.T + 1u) * subs;
+}
+
 template <bool SCATTER>
 struct KvPieces {
     static constexpr bool kTimed = false;
+    static constexpr bool kPlans = true;
     uint32_t layer0, n_layers, n, subs;
     const uint32_t *reqs, *tok_start;
     uint8_t *buf_k, *buf_v;
     unsigned long long cap_tokens, layer_stride;
-    __device__ unsigned long long total(const Geom &g) const { return (unsigned long long)n_layers * g.st->g_total_items; }
+    uint32_t *cu_out;                     // cu_seqlens for the caller (local plan only; may be null)
+    const uint32_t *cu_items, *cu_rows;   // set by plan(): shared memory, or the context's scratch
+    // Whole CTA.  `buf` holds 2 * (kLocalPlanMax + 1) words, `tmp` 32 scan words.
+    __device__ void plan(const Geom &g, uint32_t *buf, unsigned long long *tmp)
+    {
+        if (n > kLocalPlanMax) { cu_items = g.g_cu_items; cu_rows = g.g_cu_rows; return; }
+        uint32_t *rows_s = buf, *items_s = buf + kLocalPlanMax + 1;
+        const bool lead = blockIdx.x == 0;            // one CTA reports errors and writes cu_seqlens
+        unsigned long long run_rows = 0, run_items = 0, tot;
+        for (uint32_t b = 0; b < n; b += blockDim.x) {
+            const uint32_t k = b + threadIdx.x;
+            uint32_t rows = 0, items = 0;
+            if (k < n) kv_plan_entry(g, reqs, tok_start, k, subs, lead, rows, items);
+            const unsigned long long incl = block_incl_scan(((unsigned long long)items << 32) | rows, tmp, &tot);
+            if (k < n) {
+                const uint32_t ex_rows = (uint32_t)(run_rows + (uint32_t)incl - rows);
+                rows_s[k] = ex_rows;
+                items_s[k] = (uint32_t)(run_items + (uint32_t)(incl >> 32) - items);
+                if (lead && cu_out) cu_out[k] = ex_rows;
+            }
+            run_rows += (uint32_t)tot;
+            run_items += (uint32_t)(tot >> 32);
+        }
+        if (threadIdx.x == 0) {
+            rows_s[n] = (uint32_t)run_rows; items_s[n] = (uint32_t)run_items;
+            if (lead && cu_out) cu_out[n] = (uint32_t)run_rows;
+        }
+        __syncthreads();
+        cu_items = items_s; cu_rows = rows_s;
+    }
+    __device__ unsigned long long total(const Geom &) const { return (unsigned long long)n_layers * cu_items[n]; }
     __device__ Piece get(const Geom &g, unsigned long long it64) const
     {
-        const uint32_t per_layer = g.st->g_total_items;
+        const uint32_t per_layer = cu_items[n];
         const uint32_t dl = (uint32_t)(it64 / per_layer);
         const uint32_t it = (uint32_t)(it64 % per_layer);
-        const uint32_t k = find_owner(g.g_cu_items, 0u, n, 0u, it);
-        const uint32_t rel = it - g.g_cu_items[k];
-        const uint32_t row0 = g.g_cu_rows[k], rows = g.g_cu_rows[k + 1] - row0;
+        const uint32_t k = find_owner(cu_items, 0u, n, 0u, it);
+        const uint32_t rel = it - cu_items[k];
+        const uint32_t row0 = cu_rows[k], rows = cu_rows[k + 1] - row0;
         if (!SCATTER && (unsigned long long)row0 + rows > cap_tokens) {
             if (rel == 0 && dl == 0) record_error(g.st, AVMP_DEV_OUT_OVERFLOW);
             return Piece{nullptr, nullptr, 0};
@@ -277,7 +330,7 @@ struct Ring {
 constexpr int kBatch = 31;   // pieces looked up per hand-over (lanes 1..31)
 
 template <class F>
-__global__ void __launch_bounds__(kBulkThreads, kBulkCtasPerSm) stream_bulk_kernel(const Geom g, const F f)
+__global__ void __launch_bounds__(kBulkThreads, kBulkCtasPerSm) stream_bulk_kernel(const Geom g, const F f_in)
 {
     extern __shared__ __align__(1024) uint8_t ring_mem[];
     __shared__ __align__(8) unsigned long long bars[kBulkWarps * kStages];
@@ -289,6 +342,12 @@ __global__ void __launch_bounds__(kBulkThreads, kBulkCtasPerSm) stream_bulk_kern
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     pdl_prologue();
     __syncthreads();
+    F f = f_in;
+    if constexpr (F::kPlans) {
+        __shared__ uint32_t plan_buf[2 * (kLocalPlanMax + 1)];
+        __shared__ unsigned long long plan_tmp[32];
+        f.plan(g, plan_buf, plan_tmp);
+    }
     const unsigned long long total = f.total(g);
 
     // warp w of CTA c takes pieces (w * grid + c) + j * (grid * warps), j = 0, 1, ...: at any moment
@@ -337,10 +396,16 @@ __global__ void __launch_bounds__(kBulkThreads, kBulkCtasPerSm) stream_bulk_kern
 }
 
 template <class F>
-__global__ void __launch_bounds__(kGenThreads) stream_generic_kernel(const Geom g, const F f)
+__global__ void __launch_bounds__(kGenThreads) stream_generic_kernel(const Geom g, const F f_in)
 {
     const int lane = threadIdx.x & 31;
     pdl_prologue();
+    F f = f_in;
+    if constexpr (F::kPlans) {
+        __shared__ uint32_t plan_buf[2 * (kLocalPlanMax + 1)];
+        __shared__ unsigned long long plan_tmp[32];
+        f.plan(g, plan_buf, plan_tmp);
+    }
     const unsigned long long total = f.total(g);
     const unsigned long long nw = (unsigned long long)gridDim.x * (kGenThreads / 32);
     const unsigned long long it0 = (unsigned long long)(threadIdx.x >> 5) * gridDim.x + blockIdx.x;
@@ -412,18 +477,7 @@ kv_plan_kernel(const Geom g, const uint32_t *__restrict__ reqs, const uint32_t *
     for (uint32_t b = 0; b < n; b += kStepThreads) {
         const uint32_t k = b + tid;
         uint32_t rows = 0, items = 0;
-        if (k < n) {
-            const uint32_t r = reqs[k];
-            const uint32_t st = r < g.R ? g.r_state[r] : AVMP_REQ_EMPTY;
-            const uint32_t t0 = tok_start ? tok_start[k] : 0u;
-            if (st == AVMP_REQ_EMPTY) record_error(g.st, AVMP_DEV_BAD_REQUEST);
-            else {
-                const uint32_t len = g.r_len[r];
-                if (t0 > len) record_error(g.st, AVMP_DEV_BAD_REQUEST);
-                else rows = len - t0;
-            }
-            if (rows) items = ((t0 + rows - 1u) / g.T - t0 / g.T + 1u) * subs;
-        }
+        if (k < n) kv_plan_entry(g, reqs, tok_start, k, subs, true, rows, items);
         const unsigned long long incl = block_incl_scan(((unsigned long long)items << 32) | rows, tmp, &tot);
         if (k < n) {
             const uint32_t ex_rows = (uint32_t)(run_rows + (uint32_t)incl - rows);
@@ -463,12 +517,14 @@ cudaError_t launch_kv(const Geom &g, bool scatter, uint32_t layer0, uint32_t n_l
 {
     const unsigned long long part = (unsigned long long)g.T * g.row_bytes;     // K (or V) bytes of a page
     const uint32_t subs = 2u * (uint32_t)((part + kStage - 1) / kStage);
-    cudaError_t e = launch_pdl(kv_plan_kernel, dim3(1), dim3(kStepThreads), 0, l.stream, g, reqs, tok_start, n, subs, cu_out);
-    if (e != cudaSuccess) return e;
+    if (n > kLocalPlanMax) {      // long request lists: plan once, into the context's scratch
+        cudaError_t e = launch_pdl(kv_plan_kernel, dim3(1), dim3(kStepThreads), 0, l.stream, g, reqs, tok_start, n, subs, cu_out);
+        if (e != cudaSuccess) return e;
+    }
     const bool bulk_ok = mult16(g.row_bytes) && mult16(g.U[0]) && mult16(g.kv_layer_bytes) && mult16(layer_stride);
     if (scatter)
-        return launch_stream(g, KvPieces<true>{layer0, n_layers, n, subs, reqs, tok_start, (uint8_t *)k, (uint8_t *)v, cap_tokens, layer_stride}, bulk_ok, l);
-    return launch_stream(g, KvPieces<false>{layer0, n_layers, n, subs, reqs, tok_start, (uint8_t *)k, (uint8_t *)v, cap_tokens, layer_stride}, bulk_ok, l);
+        return launch_stream(g, KvPieces<true>{layer0, n_layers, n, subs, reqs, tok_start, (uint8_t *)k, (uint8_t *)v, cap_tokens, layer_stride, cu_out, nullptr, nullptr}, bulk_ok, l);
+    return launch_stream(g, KvPieces<false>{layer0, n_layers, n, subs, reqs, tok_start, (uint8_t *)k, (uint8_t *)v, cap_tokens, layer_stride, cu_out, nullptr, nullptr}, bulk_ok, l);
 }
 
 cudaError_t launch_ssm(const Geom &g, bool scatter, uint32_t layer0, uint32_t n_layers, const uint32_t *reqs, uint32_t n,

@@ -12,6 +12,7 @@ namespace avmp {
 
 constexpr uint32_t kInvalid = 0xFFFFFFFFu;
 constexpr unsigned long long kNone64 = 0xFFFFFFFFFFFFFFFFull;
+constexpr uint32_t kLocalPlanMax = 1024;    // longest request list a KV copy plans inside its own CTAs
 constexpr int kStepThreads = 1024;          // one CTA plans a step; one op per thread per window
 constexpr uint32_t kHostStepMaxOps = 65536; // staging capacity of avmp_step_host
 

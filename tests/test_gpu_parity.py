@@ -654,6 +654,39 @@ def test_edge_cases(env):
     env["same"](g, o, w, "after step_host")
 
 
+@pytest.mark.parametrize("n_list", [1024, 1025, 3000])
+def test_long_request_lists(env, n_list):
+    """KV gathers plan inside the copy kernel up to 1024 requests and through a separate plan kernel
+    beyond: a few requests repeated in a long list, on both sides of the switch, single-layer and
+    multi-layer, against the oracle."""
+    w = W.config("pr1", pool_bytes=64 * W.MiB, max_requests=3008)     # a list may not exceed the slot table
+    g, o = _pair(env, w, with_store=True)
+    h = PayloadHarness(w, [g, o], kv_layers=[0, 1, 2], ssm_layers=[1])
+    d = W.ClosedLoopDriver(w)
+
+    def step(ops):
+        so = o.step(ops)
+        assert np.array_equal(g.step(ops), so)
+        return so
+
+    W.record_trace(w, step, max_steps=40, driver=d, on_step=lambda d, a, b: h.apply_writes(d.writes))
+    run = np.flatnonzero(d.state == 1).astype(np.uint32)
+    assert len(run) >= 8
+    reqs = np.resize(run[:6], n_list).astype(np.uint32)
+    reqs[5::97] = 2000                                           # a few empty slots in between
+    total = int(o.tables()["req_len"][reqs].sum())
+    for layer in (0, 2):
+        gk, gv, gcu, gb = g.gather_kv(layer, reqs, total)
+        ok, ov, ocu, ob = o.gather_kv(layer, reqs, total)
+        assert gb == ob and np.array_equal(gcu, ocu)
+        assert np.array_equal(gk, ok) and np.array_equal(gv, ov)
+    fk, fv, fcu = g.gather_kv_layers(0, 3, reqs, total)
+    for l in range(3):
+        ok, ov, ocu, _ = o.gather_kv(l, reqs, total)
+        assert np.array_equal(fk[l, :total], ok) and np.array_equal(fv[l, :total], ov) and np.array_equal(fcu, ocu)
+    g.ctx.clear_error()
+
+
 def test_both_pools_short_in_one_op(env):
     """An admit short in both pools: SSM handler first (migrates), then the KV handler (throttled)."""
     w = W.config("tiny", pool_bytes=2048, migration_batch_size=3)
