@@ -231,7 +231,10 @@ AVMP_API int avmp_translate(avmp_ctx *ctx, const uint32_t *d_handles, uint32_t n
  * of the held lengths, n_reqs + 1 entries, always written).  Only valid tokens are copied
  * (the last page may be partial).  A slot that holds no chain contributes length 0 and a
  * sticky AVMP_DEV_BAD_REQUEST; a request whose rows would pass out_capacity_tokens copies
- * nothing (AVMP_DEV_OUT_OVERFLOW).  Output pointers must be 16-byte aligned. */
+ * nothing (AVMP_DEV_OUT_OVERFLOW).  Output pointers must be 16-byte aligned.
+ * Lists of up to 1024 requests are planned inside the copy kernel (one launch, no shared
+ * scratch); longer lists are planned by a kernel of their own into the context's workspace, so
+ * KV gathers / scatters with such lists must not overlap on the GPU (keep them on one stream). */
 AVMP_API int avmp_gather_kv(avmp_ctx *ctx, uint32_t attn_layer, const uint32_t *d_reqs, uint32_t n_reqs,
                    void *d_out_k, void *d_out_v, uint64_t out_capacity_tokens,
                    uint32_t *d_cu_seqlens, void *stream);
