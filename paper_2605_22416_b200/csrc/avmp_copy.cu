@@ -245,23 +245,41 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 // Both directions carry an L2 evict-first hint: the bytes stream through once, and keeping them
-// from displacing each other's lines was worth 2-5 % on this part.
+// from displacing each other's lines was worth 2-5 % on this part (AVMP_LOAD_HINT / AVMP_STORE_HINT = 0
+// build the unhinted forms: without the load hint the benchmark step loses 1.7 %, without the store
+// hint 0.5 %, single-layer launches 3-4 % each).
 __device__ __forceinline__ unsigned long long l2_policy_evict_first()
 {
     unsigned long long p;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
     return p;
 }
+#ifndef AVMP_LOAD_HINT
+#define AVMP_LOAD_HINT 1
+#endif
+#ifndef AVMP_STORE_HINT
+#define AVMP_STORE_HINT 1
+#endif
 __device__ __forceinline__ void bulk_g2s(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar,
                                          unsigned long long pol)
 {
+#if AVMP_LOAD_HINT
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
                  :: "r"(dst_smem), "l"(src), "r"(bytes), "r"(bar), "l"(pol) : "memory");
+#else
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
+#endif
 }
 __device__ __forceinline__ void bulk_s2g(void *dst, uint32_t src_smem, uint32_t bytes, unsigned long long pol)
 {
+#if AVMP_STORE_HINT
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;"
                  :: "l"(dst), "r"(src_smem), "r"(bytes), "l"(pol) : "memory");
+#else
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 :: "l"(dst), "r"(src_smem), "r"(bytes) : "memory");
+#endif
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
 template <int N>
