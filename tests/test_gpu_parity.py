@@ -595,15 +595,25 @@ def test_device_session_loop_matches_host_loop(env, steps, over):
     sd.close()
 
 
-def test_device_loop_replayed_from_a_cuda_graph(env):
+@pytest.mark.parametrize("kind", ["queue", "sessions"])
+def test_device_loop_replayed_from_a_cuda_graph(env, kind):
     """Fifty engine steps of the on-device loop captured once in a CUDA graph and replayed ten
     times: same final state as five hundred steps of the host loop on the oracle."""
     torch = env["torch"]
     from paper_2605_22416_b200 import binding as B
-    w = W.config("pr1", pool_bytes=40 * W.MiB, min_rebalance_interval_ops=100)
-    reqs = W.make_requests(w)
-    g = env["GpuEngine"](w)
-    dd = B.DeviceDriver(g.ctx, reqs.prompt, reqs.output, w.concurrency)
+    if kind == "queue":
+        w = W.config("pr1", pool_bytes=40 * W.MiB, min_rebalance_interval_ops=100)
+        reqs = W.make_requests(w)
+        g = env["GpuEngine"](w)
+        dd = B.DeviceDriver(g.ctx, reqs.prompt, reqs.output, w.concurrency)
+        host = dict(requests=reqs)
+    else:
+        w = W.config("agentic_burst", pool_bytes=3 * W.GiB)
+        ses = W.make_sessions(w)
+        g = env["GpuEngine"](w)
+        dd = B.SessionDriver(g.ctx, ses.arrival_step, ses.n_turns, ses.turn_prompt, ses.turn_output,
+                             ses.turn_think, w.concurrency)
+        host = dict(sessions=ses)
     torch.cuda.synchronize()
     stream = torch.cuda.Stream()
     graph = torch.cuda.CUDAGraph()
@@ -615,7 +625,7 @@ def test_device_loop_replayed_from_a_cuda_graph(env):
         graph.replay()
     torch.cuda.synchronize()
     o = env["Oracle"].from_workload(w)
-    d = W.ClosedLoopDriver(w, requests=reqs)
+    d = W.ClosedLoopDriver(w, **host)
     for _ in range(500):
         d.feed(o.step(d.next_batch()))
     env["same"](g, o, w, "graph replay vs host loop")
