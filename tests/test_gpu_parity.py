@@ -125,7 +125,7 @@ def test_longest_chain_and_full_pools(env):
     env["same"](g, o, w, "65536-op batch")
 
 
-@pytest.mark.parametrize("case", range(10))
+@pytest.mark.parametrize("case", range(int(os.environ.get("AVMP_RANDOM_CASES", "10"))))   # more cases on demand
 def test_random_shapes_and_policies(env, case):
     """Random cache shapes (rows that are and are not 16-byte multiples: both copy paths), pool
     sizes, splits, migration_batch_size, throttle and thresholds; random op batches; payload written
