@@ -697,6 +697,45 @@ def test_long_request_lists(env, n_list):
     g.ctx.clear_error()
 
 
+def test_kv_gathers_on_two_streams(env):
+    """Two KV gathers with different request lists issued on two streams (they may overlap on the GPU):
+    lists of up to 1024 requests are planned inside each launch, so the results equal the ones of the
+    same calls issued one after the other."""
+    torch = env["torch"]
+    w = W.config("short_uniform", concurrency=96)
+    g = env["GpuEngine"](w)
+    n = 90
+    lens = (np.arange(n) * 37 % 300 + 20).astype(np.uint32)
+    assert (g.step(W.make_ops(W.OP_ADMIT, np.arange(n), lens)) == 0).all()
+    dev, row = g.dev, w.model.kv_row_bytes
+    rng = np.random.default_rng(5)
+    lists = [rng.permutation(n)[:70].astype(np.uint32), rng.permutation(n)[:55].astype(np.uint32)]
+    tot = [int(lens[l].sum()) for l in lists]
+    # payload: every page of the arena gets bytes of its own
+    g.ctx.arena[:].copy_(torch.randint(0, 256, (g.ctx.arena.numel(),), dtype=torch.uint8, device=dev))
+    d_lists = [torch.from_numpy(l.view(np.int32)).to(dev) for l in lists]
+
+    def buffers():
+        return [(torch.zeros((t, row), dtype=torch.uint8, device=dev), torch.zeros((t, row), dtype=torch.uint8, device=dev),
+                 torch.zeros(len(l) + 1, dtype=torch.int32, device=dev)) for t, l in zip(tot, lists)]
+
+    ref = buffers()
+    for i in range(2):
+        g.ctx.gather_kv(i, d_lists[i], len(lists[i]), ref[i][0], ref[i][1], tot[i], ref[i][2])
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    for rep in range(20):
+        out = buffers()
+        torch.cuda.synchronize()
+        for i in range(2):
+            g.ctx.gather_kv(i, d_lists[i], len(lists[i]), out[i][0], out[i][1], tot[i], out[i][2],
+                            stream=streams[i].cuda_stream)
+        torch.cuda.synchronize()
+        for i in range(2):
+            assert all(torch.equal(a, b) for a, b in zip(out[i], ref[i])), (rep, i)
+    assert g.stats()["error_code"] == 0
+
+
 def test_both_pools_short_in_one_op(env):
     """An admit short in both pools: SSM handler first (migrates), then the KV handler (throttled)."""
     w = W.config("tiny", pool_bytes=2048, migration_batch_size=3)
