@@ -145,12 +145,22 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     ctx = B.Context.from_workload(w, device=dev)
     drv = W.ClosedLoopDriver(w)
     trace = []
+
+    def held_units():
+        # units every slot holds, from the driver's bookkeeping: pages of the chain, SSM blocks while running
+        return -(-drv.len // m.page_tokens), np.where(drv.state == 1, m.n_ssm_layers, 0)
+
     while not drv.done and drv.step < n_steps:
         ops = drv.next_batch()
         st = np.zeros(len(ops), np.uint32)
+        pages0, blocks0 = held_units()
         ctx.step_host(np.ascontiguousarray(ops), len(ops), st)
         drv.feed(st)
-        rec = {"ops": ops, "run": drv.running_slots.astype(np.uint32), "lens": drv.len[drv.running_slots].copy()}
+        pages1, blocks1 = held_units()
+        rec = {"ops": ops, "run": drv.running_slots.astype(np.uint32), "lens": drv.len[drv.running_slots].copy(),
+               # lower bound on units allocated + freed by this batch (a slot freed and re-admitted in one
+               # step counts its net change only)
+               "units": int(np.abs(pages1 - pages0).sum() + np.abs(blocks1 - blocks0).sum())}
         if drv.step > WS:
             t, _ = ctx.export_tables()
             chain = t["req_chain"].reshape(w.max_requests, w.max_pages)
@@ -344,7 +354,10 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
                    "multi_gpu": "replicas only: one independent context per GPU, no collective"},
         "allocator": {"ops_per_s": sums[1] / (sum(per["step"]) * 1e-3) * (world if world > 1 else 1),
                       "us_per_step": step_avg_ms * 1e3, "ops_per_step": n_ops_total / K,
-                      "note": "avmp_step + avmp_translate, CUDA events around the two calls, rank 0's timing"},
+                      "units_per_step": sum(r["units"] for r in timed) / K,
+                      "unit_allocs_and_frees_per_s": sum(r["units"] for r in timed) / (sum(per["step"]) * 1e-3),
+                      "note": "avmp_step + avmp_translate, CUDA events around the two calls, rank 0's timing; units = "
+                              "KV pages + SSM blocks allocated or freed, counted from the request slots' net change per step"},
         "gather_kv": {"gbs": kv_launch_bytes / (kv_avg_ms * 1e-3) / 1e9, "avg_launch_ms": kv_avg_ms,
                       "frac_of_peak": kv_launch_bytes / (kv_avg_ms * 1e-3) / 1e9 / peak,
                       "note": "avmp_gather_kv_layers: one copy launch for all attention layers (the request-list plan is computed inside it)"},
