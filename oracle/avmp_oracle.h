@@ -22,7 +22,9 @@
  * operation; gathers against a payload that is a pure function of (request,
  * token).  The free-list order, the choice of which live blocks move where and
  * the unit of migration_batch_size are policy the paper leaves open: for those
- * this file *is* the definition (parity unpinned by the paper).
+ * this file *is* the definition (parity unpinned by the paper).  The reclaim_gap
+ * option is a variant of the waste rule that the paper does not have; it is pinned
+ * by its own hand-worked trace, a closed-form case and the two separate models.
  */
 #ifndef AVMP_ORACLE_H
 #define AVMP_ORACLE_H
