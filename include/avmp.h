@@ -298,7 +298,11 @@ AVMP_API int avmp_get_stats(avmp_ctx *ctx, avmp_stats *h_out, void *stream);
 /* Clear the sticky device error code and count.  Stream-ordered. */
 AVMP_API int avmp_clear_error(avmp_ctx *ctx, void *stream);
 
-/* Tables <-> host (parity checks, snapshot / restore).  Both synchronise the stream. */
+/* Tables <-> host (parity checks, snapshot / restore).  Both synchronise the stream.
+ * Import checks the snapshot on the host first (capacities and pool-byte conservation, free lists
+ * distinct and inside their stores, page table and owner table mutually inverse, every handle of
+ * every request resolvable and owned once) and returns AVMP_EINVAL, with the context untouched, if
+ * it does not hang together: the kernels index these tables without bounds checks. */
 AVMP_API int avmp_export_tables(avmp_ctx *ctx, avmp_tables *h_out, void *stream);
 AVMP_API int avmp_import_tables(avmp_ctx *ctx, const avmp_tables *h_in, void *stream);
 

@@ -5,6 +5,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "avmp_dev.cuh"
 
@@ -81,6 +82,75 @@ void fill_stats(const avmp_ctx *c, const DevState &d, avmp_stats *o)
     o->step_ns_total = (uint64_t)(d.cyc_total * ns_per_cycle);
     o->step_ns_oom_retry = (uint64_t)(d.cyc_oom * ns_per_cycle);
     o->step_ns_migration_plan = (uint64_t)(d.cyc_mig * ns_per_cycle);
+}
+
+// A snapshot is accepted only if the kernels could have produced it: they index the tables
+// without bounds checks, so a table that does not hang together must never reach the device.
+bool tables_consistent(const avmp_ctx *c, const avmp_tables *t)
+{
+    const Geom &g = c->g;
+    const avmp_stats &st = t->stats;
+    if (st.fsm_state > AVMP_FSM_REBALANCING) return false;
+    if (st.last_rebalance_op != kNone64 && st.last_rebalance_op > st.op_counter) return false;
+    unsigned __int128 bytes = st.gap_bytes;
+    for (int p = 0; p < 2; ++p) {
+        if (st.cap[p] > g.V[p]) return false;
+        bytes += (unsigned __int128)st.cap[p] * g.U[p];
+    }
+    if (bytes != g.P_al) return false;                         // pool bytes are conserved
+    uint64_t live[2] = {0, 0};
+    std::vector<uint8_t> mark;
+    for (int p = 0; p < 2; ++p) {
+        const uint32_t V = g.V[p], cap = (uint32_t)st.cap[p], nf = t->n_slot_stack[p], nv = t->n_vid_stack[p];
+        const uint32_t *S = t->slot_stack[p], *W = t->vid_stack[p], *VT = t->vt[p], *OW = t->ow[p];
+        if (nf > cap || nv > V) return false;
+        mark.assign(V, 0);
+        for (uint32_t i = 0; i < nf; ++i) {                    // free slots: inside the store, distinct
+            if (S[i] >= cap || mark[S[i]]) return false;
+            mark[S[i]] = 1;
+        }
+        for (uint32_t s = 0; s < V; ++s) {                     // owned slots: not free, mapped back by their id
+            const uint32_t v = OW[s];
+            if (v == kInvalid) continue;
+            if (s >= cap || mark[s] || v >= V || VT[v] != s) return false;
+            live[p] += 1;
+        }
+        if (live[p] != (uint64_t)cap - nf) return false;
+        mark.assign(V, 0);
+        for (uint32_t i = 0; i < nv; ++i) {                    // free ids: distinct, unmapped
+            if (W[i] >= V || mark[W[i]] || VT[W[i]] != kInvalid) return false;
+            mark[W[i]] = 1;
+        }
+        uint64_t mapped = 0;
+        for (uint32_t v = 0; v < V; ++v) {
+            if (VT[v] == kInvalid) continue;
+            if (VT[v] >= cap || OW[VT[v]] != v) return false;
+            mapped += 1;
+        }
+        if (mapped != live[p] || (uint64_t)nv != (uint64_t)V - live[p]) return false;
+    }
+    // every live unit belongs to exactly one request
+    std::vector<uint8_t> ref[2];
+    ref[0].assign(g.V[0], 0); ref[1].assign(g.V[1], 0);
+    uint64_t held[2] = {0, 0};
+    for (uint32_t r = 0; r < g.R; ++r) {
+        const uint32_t state = t->req_state[r], np = t->req_npages[r], len = t->req_len[r];
+        if (state == AVMP_REQ_EMPTY) { if (np || len) return false; continue; }
+        if (state != AVMP_REQ_LIVE && state != AVMP_REQ_KV_ONLY) return false;
+        if (np > g.max_pages || ((uint64_t)len + g.T - 1) / g.T != np) return false;
+        for (uint32_t j = 0; j < np; ++j) {
+            const uint32_t h = t->req_chain[(size_t)r * g.max_pages + j], v = h & 0x7FFFFFFFu;
+            if ((h >> 31) != AVMP_POOL_KV || v >= g.V[0] || t->vt[0][v] == kInvalid || ref[0][v]) return false;
+            ref[0][v] = 1; held[0] += 1;
+        }
+        if (state == AVMP_REQ_LIVE)
+            for (uint32_t l = 0; l < g.ns; ++l) {
+                const uint32_t h = t->req_ssm[(size_t)r * g.ns + l], v = h & 0x7FFFFFFFu;
+                if ((h >> 31) != AVMP_POOL_SSM || v >= g.V[1] || t->vt[1][v] == kInvalid || ref[1][v]) return false;
+                ref[1][v] = 1; held[1] += 1;
+            }
+    }
+    return held[0] == live[0] && held[1] == live[1];
 }
 
 }  // namespace
@@ -408,6 +478,7 @@ int avmp_import_tables(avmp_ctx *c, const avmp_tables *t, void *stream)
         if (t->n_slot_stack[p] > g.V[p] || t->n_vid_stack[p] > g.V[p] || t->stats.cap[p] > g.V[p]) return AVMP_EINVAL;
     }
     if (!t->req_state || !t->req_len || !t->req_npages || !t->req_chain || (g.ns && !t->req_ssm)) return AVMP_EINVAL;
+    if (!tables_consistent(c, t)) return AVMP_EINVAL;          // nothing has been copied yet
     bool ok = true;
     auto push = [&](uint32_t *dst, const uint32_t *src, size_t n) {
         if (n) ok = ok && cudaMemcpyAsync(dst, src, n * 4, cudaMemcpyHostToDevice, s) == cudaSuccess;

@@ -797,3 +797,58 @@ def test_export_import_roundtrip(env):
 
     W.record_trace(w, step2, max_steps=200, driver=d)
     env["same"](g2, o, w, "after more steps")
+
+
+def test_import_rejects_inconsistent_snapshots(env):
+    """A snapshot that the kernels could not have produced is refused on the host and the context stays
+    as it was: the kernels index the tables without bounds checks."""
+    from paper_2605_22416_b200.binding import AvmpError
+    w = W.config("pr1", pool_bytes=24 * W.MiB, concurrency=12, min_rebalance_interval_ops=50,
+                 migration_batch_size=6, n_requests=60)
+    g, o = _pair(env, w)
+    d = W.ClosedLoopDriver(w)
+
+    def step(ops):
+        so = o.step(ops)
+        assert np.array_equal(g.step(ops), so)
+        return so
+
+    W.record_trace(w, step, max_steps=120, driver=d)
+    good_t, good_s = g.ctx.export_tables()
+    assert good_s["n_rebalance"] > 0 and (good_t["req_state"] == 1).sum() >= 4
+    live = int(np.flatnonzero(good_t["req_state"] == 1)[0])
+    mp, ns = g.max_pages, w.model.n_ssm_layers
+
+    def variant(f_tables=None, f_stats=None):
+        t = {k: v.copy() for k, v in good_t.items()}
+        s = dict(good_s)
+        if f_tables: f_tables(t)
+        if f_stats: f_stats(s)
+        return t, s
+
+    def set_(key, idx, val):
+        def f(t): t[key][idx] = val
+        return f
+
+    bad = {
+        "free slot beyond the store": variant(set_("slot_stack_kv", 0, good_s["cap_kv"])),
+        "free slot twice": variant(set_("slot_stack_ssm", 0, int(good_t["slot_stack_ssm"][1]))),
+        "chain handle beyond the id space": variant(set_("req_chain", live * mp, good_s["vid_space_kv"] + 5)),
+        "chain handle of a free id": variant(set_("req_chain", live * mp, int(good_t["vid_stack_kv"][0]))),
+        "chain handle with the SSM tag": variant(set_("req_chain", live * mp, int(good_t["req_chain"][live * mp]) | (1 << 31))),
+        "SSM handle held twice": variant(set_("req_ssm", live * ns, int(good_t["req_ssm"][live * ns + 1]))),
+        "page table entry beyond the store": variant(set_("vt_kv", int(good_t["req_chain"][live * mp]), good_s["cap_kv"] + 1)),
+        "owner table not the inverse": variant(set_("ow_ssm", int(good_t["vt_ssm"][int(good_t["req_ssm"][live * ns]) & 0x7FFFFFFF]), 0x12345)),
+        "length does not match the pages": variant(set_("req_len", live, int(good_t["req_len"][live]) + 64)),
+        "unknown request state": variant(set_("req_state", live, 7)),
+        "capacity does not conserve the pool": variant(None, lambda s: s.__setitem__("cap_kv", s["cap_kv"] + 1)),
+        "last rebalance in the future": variant(None, lambda s: s.__setitem__("last_rebalance_op", s["op_counter"] + 9)),
+    }
+    for what, (t, s) in bad.items():
+        with pytest.raises(AvmpError):
+            g.ctx.import_tables(t, s)
+        env["same"](g, o, w, f"context untouched after: {what}")
+    g.ctx.import_tables(good_t, good_s)                     # the unmodified snapshot goes in
+    env["same"](g, o, w, "after importing the good snapshot")
+    ops = d.next_batch()
+    assert np.array_equal(g.step(ops), o.step(ops))
