@@ -130,7 +130,8 @@ __global__ void __launch_bounds__(kStepThreads, 1) sess_build_kernel(const Sess 
             if (s == forced) fin = 1;
             else if (state == RUNNING_) {
                 fin = d.slot_rem[s] == 0 ? 1u : 0u; ext = 1u - fin;
-                if (fin && d.slot_turn[s] + 1u < d.n_turns[d.slot_uid[s]]) flags = AVMP_FLAG_KEEP_KV;
+                // (a turn count beyond max_turns is cut there: the per-turn arrays have max_turns columns)
+                if (fin && d.slot_turn[s] + 1u < min(d.n_turns[d.slot_uid[s]], MT)) flags = AVMP_FLAG_KEEP_KV;
             } else if (state == FREE_) fre = 1;
         }
         const unsigned long long v = (unsigned long long)fin | ((unsigned long long)ext << 21) | ((unsigned long long)fre << 42);
