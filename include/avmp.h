@@ -349,7 +349,8 @@ AVMP_API int avmp_driver_export(avmp_driver *drv, uint32_t *h_state, uint32_t *h
  * request, an admit that fails with nothing running and nothing parked is dropped.
  * All five arrays are device arrays of uint32 owned by the caller and must outlive the driver;
  * concurrency <= 1024.  The workspace (avmp_session_driver_workspace_bytes, 256-byte aligned) is
- * the caller's.  Each step is a few stream-ordered launches with no host round trip. */
+ * the caller's.  Each step is one launch plus the relocation copy (a few launches when a batch may
+ * hold more than one migration), with no host round trip. */
 typedef struct avmp_session_driver avmp_session_driver;
 typedef struct {
     uint64_t steps, completed, dropped, preempted, evicted, n_oom_admit, n_oom_extend;

@@ -39,6 +39,7 @@ struct SessState {
     uint32_t n_fin, n_ext, n_adm, n_ops;
     uint32_t took_front, took_rq, took_back, break_uid;   // what the batch builder removed from the queues
     uint32_t starved;                 // the batch left an entry without a slot
+    uint32_t hi;                      // slots >= hi have never been used: the scans stop there
 };
 
 struct Sess {
@@ -65,7 +66,7 @@ struct SessShared {
     unsigned long long tmp[32];
     uint32_t tmp32[32];
     SessState st;
-    uint32_t s_completed, s_evicted, s_ext_ok, s_ext_oom, s_has_pre, s_pre_uid, s_n_parked;
+    uint32_t s_completed, s_evicted, s_ext_ok, s_ext_oom, s_has_pre, s_pre_uid, s_n_parked, s_hi;
     unsigned long long s_oldest_parked, s_newest_running;
 };
 
@@ -88,11 +89,9 @@ __global__ void __launch_bounds__(kStepThreads, 1) sess_init_kernel(const Sess d
     }
 }
 
-// Build the next batch.
-__global__ void __launch_bounds__(kStepThreads, 1) sess_build_kernel(const Sess d)
+// Build the next batch (whole CTA; blockDim.x >= concurrency).
+__device__ void sess_build_body(const Sess &d, SessShared &sm)
 {
-    __shared__ SessShared sm;
-    pdl_prologue();
     unsigned long long *tmp = sm.tmp;
     SessState &st = sm.st;
     const uint32_t tid = threadIdx.x, NT = blockDim.x;
@@ -122,10 +121,11 @@ __global__ void __launch_bounds__(kStepThreads, 1) sess_build_kernel(const Sess 
 
     // FINISH, EXTEND and free slots, ascending (three counters packed 21 bits each)
     unsigned long long run = 0;
-    for (uint32_t b = 0; b < R; b += NT) {
+    const uint32_t hi = st.hi;                 // <= R; every slot at or above it is free
+    for (uint32_t b = 0; b < hi; b += NT) {
         const uint32_t s = b + tid;
         uint32_t fin = 0, ext = 0, fre = 0, flags = 0;
-        if (s < R) {
+        if (s < hi) {
             const uint32_t state = d.slot_state[s];
             if (s == forced) fin = 1;
             else if (state == RUNNING_) {
@@ -143,7 +143,8 @@ __global__ void __launch_bounds__(kStepThreads, 1) sess_build_kernel(const Sess 
     }
     __syncthreads();
     const uint32_t n_fin = (uint32_t)(run & 0x1FFFFFu), n_ext = (uint32_t)((run >> 21) & 0x1FFFFFu);
-    const uint32_t n_free = (uint32_t)((run >> 42) & 0x1FFFFFu);
+    const uint32_t n_free_lo = (uint32_t)((run >> 42) & 0x1FFFFFu);   // free slots below hi, listed
+    const uint32_t n_free = n_free_lo + (R - hi);                      // plus the untouched ones above
     uint32_t budget = st.concurrency > n_ext ? st.concurrency - n_ext : 0u;
     budget = min(budget, st.window);            // <= concurrency <= NT: one candidate per thread
 
@@ -170,7 +171,7 @@ __global__ void __launch_bounds__(kStepThreads, 1) sess_build_kernel(const Sess 
     for (uint32_t j = tid; j < n_ext; j += NT) put_op(d.ops + n_fin + j, AVMP_OP_EXTEND, 0, d.ext_slots[j], 1);
     if (tid < n_adm) {
         const uint32_t own = d.e_slot[uid];
-        const uint32_t slot = needs_free ? d.free_slots[rank] : own;
+        const uint32_t slot = needs_free ? (rank < n_free_lo ? d.free_slots[rank] : hi + (rank - n_free_lo)) : own;
         put_op(d.ops + n_fin + n_ext + tid, AVMP_OP_ADMIT, needs_free ? 0u : (uint32_t)AVMP_FLAG_RESUME, slot, d.e_prompt[uid]);
         d.adm_uid[tid] = uid; d.adm_slot[tid] = slot; d.adm_res[tid] = 1u - needs_free;
     }
@@ -188,13 +189,12 @@ __global__ void __launch_bounds__(kStepThreads, 1) sess_build_kernel(const Sess 
         o->n_fin = n_fin; o->n_ext = n_ext; o->n_adm = n_adm; o->n_ops = n_fin + n_ext + n_adm;
         *d.n_ops_word = n_fin + n_ext + n_adm;
     }
+    __syncthreads();
 }
 
-// Fold the statuses of the batch back into the slots and the queues.
-__global__ void __launch_bounds__(kStepThreads, 1) sess_feed_kernel(const Sess d)
+// Fold the statuses of the batch back into the slots and the queues (whole CTA).
+__device__ void sess_feed_body(const Sess &d, SessShared &sm)
 {
-    __shared__ SessShared sm;
-    pdl_prologue();
     unsigned long long *tmp = sm.tmp;
     SessState &st = sm.st;
     const uint32_t tid = threadIdx.x, NT = blockDim.x;
@@ -202,6 +202,7 @@ __global__ void __launch_bounds__(kStepThreads, 1) sess_feed_kernel(const Sess d
         st = *d.st;
         sm.s_completed = sm.s_evicted = sm.s_ext_ok = sm.s_ext_oom = sm.s_has_pre = sm.s_n_parked = 0;
         sm.s_pre_uid = kInvalid;
+        sm.s_hi = st.hi;
         sm.s_oldest_parked = ~0ull; sm.s_newest_running = 0ull;
     }
     __syncthreads();
@@ -256,13 +257,15 @@ __global__ void __launch_bounds__(kStepThreads, 1) sess_feed_kernel(const Sess d
         d.slot_state[s] = RUNNING_; d.slot_uid[s] = u; d.slot_len[s] = base + d.e_prompt[u];
         d.slot_rem[s] = d.e_output[u]; d.slot_turn[s] = d.e_turn[u];
         d.slot_seq[s] = st.seq + n_park + (uint32_t)ex + 1u;
+        atomicMax(&sm.s_hi, s + 1u);
     }
     __syncthreads();
+    const uint32_t new_hi = sm.s_hi;
     // who is parked, who runs: the longest-parked chain and the most recently admitted request
     {
         unsigned long long oldest = ~0ull, newest = 0ull;
         uint32_t cnt = 0;
-        for (uint32_t s = tid; s < st.R; s += NT) {
+        for (uint32_t s = tid; s < new_hi; s += NT) {
             const uint32_t state = d.slot_state[s];
             if (state == PARKED_) { cnt += 1; oldest = min(oldest, ((unsigned long long)d.slot_pseq[s] << 32) | s); }
             else if (state == RUNNING_) newest = max(newest, ((unsigned long long)d.slot_seq[s] << 32) | s);
@@ -332,8 +335,38 @@ __global__ void __launch_bounds__(kStepThreads, 1) sess_feed_kernel(const Sess d
         if ((oom_seen || st.starved) && n_parked > 0) { n.forced_slot = (uint32_t)(sm.s_oldest_parked & 0xFFFFFFFFull); n.forced_why = WHY_EVICT; }
         else if (!progress && n_running > 0 && st.n_ops > 0) { n.forced_slot = (uint32_t)(sm.s_newest_running & 0xFFFFFFFFull); n.forced_why = WHY_PREEMPT; }
         n.break_uid = kInvalid; n.starved = 0;
+        n.hi = new_hi;
         *d.st = n;
     }
+}
+
+__global__ void __launch_bounds__(kStepThreads, 1) sess_build_kernel(const Sess d)
+{
+    __shared__ SessShared sm;
+    pdl_prologue();
+    sess_build_body(d, sm);
+}
+
+__global__ void __launch_bounds__(kStepThreads, 1) sess_feed_kernel(const Sess d)
+{
+    __shared__ SessShared sm;
+    pdl_prologue();
+    sess_feed_body(d, sm);
+}
+
+// One engine step in one launch: build, allocator update, fold back.  Usable when the batch can hold
+// at most one migration (a second one needs the first one's relocation copy, a separate wide kernel).
+template <int NT>
+__global__ void __launch_bounds__(NT, 1) sess_fused_kernel(const Sess d, const Geom g)
+{
+    __shared__ SessShared sm;
+    __shared__ stepimpl::Shared<NT> sh;
+    pdl_prologue();
+    sess_build_body(d, sm);
+    const uint32_t n_ops = *d.n_ops_word;
+    stepimpl::step_body<NT>(g, sh, d.ops, n_ops, d.status, 1);
+    __syncthreads();
+    sess_feed_body(d, sm);
 }
 
 constexpr size_t kAlign = 256;
@@ -366,7 +399,7 @@ inline cudaStream_t S(void *s) { return reinterpret_cast<cudaStream_t>(s); }
 struct avmp_session_driver {
     Sess d;
     avmp_ctx *ctx;
-    uint32_t R, n_sessions, max_ops;
+    uint32_t R, n_sessions, max_ops, concurrency;
 };
 
 extern "C" {
@@ -410,7 +443,7 @@ AVMP_API int avmp_session_driver_create(avmp_session_driver **out, avmp_ctx *ctx
     d.new_key = u64(l.new_key); d.new_uid = u32(l.new_uid);
     d.ops = reinterpret_cast<avmp_op *>(b + l.ops);
     d.status = u32(l.status); d.n_ops_word = u32(l.n_ops);
-    dr->ctx = ctx; dr->R = R; dr->n_sessions = n_sessions;
+    dr->ctx = ctx; dr->R = R; dr->n_sessions = n_sessions; dr->concurrency = concurrency;
     // at most `concurrency` requests run, one more slot may be evicted, at most `concurrency` are admitted
     dr->max_ops = 2 * concurrency + 1 < 2 * R ? 2 * concurrency + 1 : 2 * R;
     SessState init;
@@ -433,6 +466,23 @@ AVMP_API int avmp_session_driver_step(avmp_session_driver *dr, void *stream)
 {
     if (!dr) return AVMP_EINVAL;
     avmp_ctx *c = dr->ctx;
+    const bool mig = c->opt.migration_enabled != 0;
+    const uint64_t rounds = mig ? (uint64_t)(dr->max_ops - 1) / c->opt.min_rebalance_interval_ops + 1 : 1;
+    if (rounds == 1) {
+        // the planning block needs a thread per admission candidate and per op of a window
+        const uint32_t need = dr->max_ops > dr->concurrency ? dr->max_ops : dr->concurrency;
+        cudaError_t e;
+        if (need <= 256) e = launch_pdl(sess_fused_kernel<256>, dim3(1), dim3(256), 0, S(stream), dr->d, c->g);
+        else if (need <= 512) e = launch_pdl(sess_fused_kernel<512>, dim3(1), dim3(512), 0, S(stream), dr->d, c->g);
+        else e = launch_pdl(sess_fused_kernel<1024>, dim3(1), dim3(1024), 0, S(stream), dr->d, c->g);
+        if (e != cudaSuccess) return AVMP_ECUDA;
+        c->launches += 1;
+        if (mig) {
+            if (launch_relocate(c->g, Launch{S(stream), c->n_sms, c->device}) != cudaSuccess) return AVMP_ECUDA;
+            c->launches += 1;
+        }
+        return AVMP_OK;
+    }
     if (launch_pdl(sess_build_kernel, dim3(1), dim3(kStepThreads), 0, S(stream), dr->d) != cudaSuccess) return AVMP_ECUDA;
     const int rc = avmp_step_indirect(c, dr->d.ops, dr->d.n_ops_word, dr->max_ops, dr->d.status, stream);
     if (rc != AVMP_OK) return rc;
