@@ -18,5 +18,11 @@ int main(void)
            (unsigned long long)l.unit_bytes[1], (unsigned long long)l.cap0[0], (unsigned long long)l.cap0[1]);
     printf("workspace_bytes=%llu\n", (unsigned long long)avmp_workspace_bytes(&m, 4ull << 30, &o));
     printf("%s\n", avmp_error_string(AVMP_ENOSPC));
+    /* struct sizes as this compiler sees them: the Python binding must declare the same */
+    printf("sizeof avmp_model_spec=%u avmp_options=%u avmp_op=%u avmp_layout=%u avmp_stats=%u avmp_tables=%u "
+           "avmp_driver_stats=%u avmp_session_stats=%u\n",
+           (unsigned)sizeof(avmp_model_spec), (unsigned)sizeof(avmp_options), (unsigned)sizeof(avmp_op),
+           (unsigned)sizeof(avmp_layout), (unsigned)sizeof(avmp_stats), (unsigned)sizeof(avmp_tables),
+           (unsigned)sizeof(avmp_driver_stats), (unsigned)sizeof(avmp_session_stats));
     return 0;
 }

@@ -45,6 +45,14 @@ def test_public_header_is_plain_c():
     out = subprocess.check_output([str(exe)]).decode()
     exe.unlink()
     assert "U_kv=262144 U_ssm=622592 kv_cap=8192 ssm_cap=3449" in out and "workspace_bytes=" in out
+    # the ctypes declarations of the binding have the sizes the C compiler gives the header's structs
+    # (the binding module needs no GPU to import; only its structure classes are used here)
+    from paper_2605_22416_b200 import binding as B
+    sizes = dict(kv.split("=") for kv in re.search(r"sizeof (.*)", out).group(1).split())
+    from paper_2605_22416_b200 import workloads as W
+    for name, n in sizes.items():
+        mine = W.OP_DTYPE.itemsize if name == "avmp_op" else ctypes.sizeof(getattr(B, name))   # ops travel as a numpy record
+        assert mine == int(n), (name, n, mine)
 
 
 def test_binding_declares_every_symbol():
