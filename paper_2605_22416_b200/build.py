@@ -13,7 +13,7 @@ CSRC = PKG / "csrc"
 LIB = Path(os.environ["AVMP_LIB"]) if os.environ.get("AVMP_LIB") else PKG / "libavmp.so"
 SOURCES = ["avmp_api.cu", "avmp_step.cu", "avmp_copy.cu", "avmp_noalloc.cu", "avmp_driver.cu",
            "avmp_sessions.cu"]
-HEADERS = [CSRC / "avmp_dev.cuh", ROOT / "include" / "avmp.h"]
+HEADERS = [CSRC / "avmp_dev.cuh", CSRC / "avmp_step_body.cuh", ROOT / "include" / "avmp.h"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--shared", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden",
               "-cudart", "static", f"-I{ROOT / 'include'}", f"-I{CSRC}"]
