@@ -547,7 +547,7 @@ def test_device_closed_loop_matches_host_loop(env, name, steps, over):
 
 
 @pytest.mark.parametrize("steps,over", [
-    (1500, {}),
+    (20_000, {}),                                                         # the whole arrival horizon
     (1200, dict(pool_bytes=3 * W.GiB)),                                  # tight: evictions, failed resumes
     (900, dict(pool_bytes=2 * W.GiB, concurrency=64, split=0.3)),         # pre-emptions, no free slot
     (700, dict(pool_bytes=3 * W.GiB, max_requests=96, concurrency=96)),   # slots run out before memory
@@ -558,7 +558,7 @@ def test_device_session_loop_matches_host_loop(env, steps, over):
     """The on-device scheduler for multi-turn sessions (arrivals, parking with KEEP_KV, resume after the
     think time, eviction of the longest-parked chain, pre-emption, drops) against the host-side batch
     builder running on the oracle: allocator tables and counters, every slot, both queues in order and
-    every scheduler counter, compared every 100 steps."""
+    every scheduler counter, compared every 100 steps (every 1000 on the long run)."""
     from paper_2605_22416_b200 import binding as B
     w = W.config("agentic_burst", **over)
     ses = W.make_sessions(w)
@@ -569,7 +569,7 @@ def test_device_session_loop_matches_host_loop(env, steps, over):
     d = W.ClosedLoopDriver(w, sessions=ses)
     done = 0
     while done < steps:
-        n = min(100, steps - done)
+        n = min(100 if steps <= 2000 else 1000, steps - done)
         for _ in range(n):
             sd.step()
             d.feed(o.step(d.next_batch()))
