@@ -546,6 +546,39 @@ def test_device_closed_loop_matches_host_loop(env, name, steps, over):
     dd.close()
 
 
+@pytest.mark.parametrize("name,over,n_requests", [
+    ("pr1", {}, None),
+    ("short_uniform", {}, None),
+    ("mixed_long", dict(migration_batch_size=16), None),
+    ("scale", {}, 60_000),
+])
+def test_device_loop_whole_traces(env, name, over, n_requests):
+    """The on-device loop run until its request list is exhausted (config 5: its first 60 000 requests),
+    step for step beside the host loop on the oracle: counters every 5000 steps, everything at the end."""
+    from paper_2605_22416_b200 import binding as B
+    w = W.config(name, **over)
+    reqs = W.make_requests(w, n_requests) if n_requests else W.make_requests(w)
+    g, o = _pair(env, w)
+    dd = B.DeviceDriver(g.ctx, reqs.prompt, reqs.output, w.concurrency)
+    d = W.ClosedLoopDriver(w, requests=reqs)
+    n = 0
+    while not d.done:
+        dd.step()
+        d.feed(o.step(d.next_batch()))
+        n += 1
+        if n % 5000 == 0:
+            ds = dd.stats()
+            assert (ds["completed"], ds["preempted"], ds["dropped"]) == (d.completed, d.preempted, d.dropped), n
+            env["same"](g, o, w, f"{name} at step {n}")
+    ds = dd.stats()
+    assert (ds["completed"], ds["preempted"], ds["dropped"]) == (d.completed, d.preempted, d.dropped)
+    assert ds["n_oom_admit"] == d.n_oom_admit and ds["n_oom_extend"] == d.n_oom_extend and ds["overflow"] == 0
+    assert d.completed + d.dropped == len(reqs.prompt) and ds["steps"] == n
+    env["same"](g, o, w, f"{name} end of trace")
+    assert (dd.export()["state"] == 0).all() and g.stats()["error_code"] == 0
+    dd.close()
+
+
 @pytest.mark.parametrize("steps,over", [
     (20_000, {}),                                                         # the whole arrival horizon
     (1200, dict(pool_bytes=3 * W.GiB)),                                  # tight: evictions, failed resumes
