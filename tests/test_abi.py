@@ -127,3 +127,18 @@ def test_replica_reduction_over_two_gloo_ranks(tmp_path):
     outs = [p.communicate(timeout=120)[0].decode() for p in procs]
     assert all(p.returncode == 0 for p in procs), outs
     assert all("ok" in o for o in outs)
+
+
+def test_plain_cuda_caller_compiles_and_links():
+    """The CUDA-runtime-only caller of the ABI builds against the header and the library here (no GPU
+    needed to compile; the GPU test runs it)."""
+    import shutil
+    from paper_2605_22416_b200 import build
+    lib = build.build_library()
+    nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
+    exe = Path(os.environ.get("TMPDIR", "/tmp")) / f"avmp_plain_cuda_caller_build_{os.getpid()}"
+    subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-std=c++17", f"-I{ROOT / 'include'}",
+                           str(ROOT / "tests" / "plain_cuda_caller.cu"), "-o", str(exe), str(lib),
+                           "-Xlinker", f"-rpath={lib.parent}"])
+    assert exe.exists()
+    exe.unlink()
