@@ -32,10 +32,11 @@ from paper_2605_22416_b200 import workloads as W  # noqa: E402
 
 METRIC = "paged gather+migration GB/s over whole engine steps (allocator ops/s reported beside it)"
 WARM_STEPS = 600          # closed-loop steps before the measured window (steady state)
-# DRAM bytes (read + write) per launch of the dominant kernel divided by its algorithmic bytes, from the
-# ncu capture summarised in profiles/ssm_gather_fused_jamba_like.md (a smaller case of the same kernel:
-# 1.04 GB per launch instead of 6.8 GB; traffic grows in proportion to the blocks gathered).
-NCU_TRAFFIC_RATIO = 0.951
+# DRAM bytes (read + write) per launch of the dominant kernel divided by its algorithmic bytes, from an ncu
+# capture of this benchmark's own launches (profiles/bench_short_uniform_dram_traffic.md; the two byte counters
+# take one pass, so the full-size launches can be captured).  Reads equal the algorithmic bytes; the last
+# 0.7 % of the writes is still in L2 when the kernel ends.  A 1 GB launch of the same kernel reads 0.953.
+NCU_TRAFFIC_RATIO = 0.993
 
 
 def _peaks():
