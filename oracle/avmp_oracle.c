@@ -343,7 +343,7 @@ uint32_t orc_gather_kv(const orc_ctx *c, uint32_t layer, const uint32_t *reqs, u
         uint32_t r = reqs[k];
         uint32_t len = holds_kv(c, r) ? c->r_len[r] : 0;
         if (!holds_kv(c, r)) ++bad;
-        else if (len > 0 && cu + len > capacity_tokens) ++bad;   /* no rows, nothing to overflow */
+        else if (cu + len > capacity_tokens) ++bad;   /* a held request has len >= 1: ADMIT / EXTEND take tokens >= 1 */
         else
             for (uint32_t t = 0; t < len; ++t) {
                 memcpy((uint8_t *)out_k + (cu + t) * row, kv_row(c, r, layer, 0, t), row);
@@ -438,6 +438,13 @@ void orc_get_stats(const orc_ctx *c, orc_stats *s)
     s->fsm_state = c->fsm;
     s->n_invalid = c->n_invalid;
     s->pool_bytes_aligned = c->P_al;
+}
+
+const uint8_t *orc_store_bytes(const orc_ctx *c, int pool, uint64_t offset, uint64_t n)
+{
+    if (pool < 0 || pool > 1 || !c->store[pool]) return NULL;
+    if (offset > c->store_bytes[pool] || n > c->store_bytes[pool] - offset) return NULL;
+    return c->store[pool] + offset;
 }
 
 const uint32_t *orc_table(const orc_ctx *c, int which, uint64_t *count)

@@ -20,7 +20,8 @@
  * model written separately (the paper's static-equivalence claim, Section 1.1);
  * a naive list-based model on tiny inputs; structural invariants after every
  * operation; gathers against a payload that is a pure function of (request,
- * token).  The free-list order, the choice of which live blocks move where and
+ * token); the position of every byte inside a unit ([layer][K, V][token][head][dim]
+ * for a page, state then window for a block) read from the raw store bytes.  The free-list order, the choice of which live blocks move where and
  * the unit of migration_batch_size are policy the paper leaves open: for those
  * this file *is* the definition (parity unpinned by the paper).  The reclaim_gap
  * option is a variant of the waste rule that the paper does not have; it is pinned
@@ -118,6 +119,11 @@ uint32_t orc_scatter_ssm(orc_ctx *c, uint32_t layer, const uint32_t *reqs, uint3
                          const void *in_state, const void *in_conv);
 
 void orc_get_stats(const orc_ctx *c, orc_stats *out);
+
+/* Read-only view of n raw bytes of a store (pool ORC_KV or ORC_SSM) starting at byte `offset`
+ * of that store, i.e. at the offsets orc_translate returns.  NULL without payload stores or when
+ * the range leaves the store.  Lets a test look at where inside a unit each byte was put. */
+const uint8_t *orc_store_bytes(const orc_ctx *c, int pool, uint64_t offset, uint64_t n);
 
 /* Views of the internal tables (owned by the context; valid until the next call). */
 enum {

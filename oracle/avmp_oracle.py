@@ -82,6 +82,8 @@ def lib():
         L.orc_scatter_ssm.restype = C.c_uint32
         L.orc_scatter_ssm.argtypes = [vp, C.c_uint32, vp, C.c_uint32, vp, vp]
         L.orc_get_stats.argtypes = [vp, vp]
+        L.orc_store_bytes.restype = C.POINTER(C.c_uint8)
+        L.orc_store_bytes.argtypes = [vp, C.c_int, C.c_uint64, C.c_uint64]
         L.orc_table.restype = u32p
         L.orc_table.argtypes = [vp, C.c_int, u64p]
         _lib = L
@@ -176,6 +178,13 @@ class Oracle:
         buf = np.zeros(len(STAT_FIELDS), np.uint64)
         lib().orc_get_stats(self._h, _ptr(buf))
         return {k: int(v) for k, v in zip(STAT_FIELDS, buf)}
+
+    def store_bytes(self, pool: int, offset: int, n: int) -> np.ndarray:
+        """Copy of n raw bytes of a store, starting at a byte offset inside that store."""
+        p = lib().orc_store_bytes(self._h, pool, offset, n)
+        if not p:
+            raise ValueError("no payload store, or the range leaves the store")
+        return np.ctypeslib.as_array(p, shape=(n,)).copy()
 
     def table(self, name: str) -> np.ndarray:
         cnt = C.c_uint64(0)

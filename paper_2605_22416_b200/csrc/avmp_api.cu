@@ -137,7 +137,8 @@ bool tables_consistent(const avmp_ctx *c, const avmp_tables *t)
         const uint32_t state = t->req_state[r], np = t->req_npages[r], len = t->req_len[r];
         if (state == AVMP_REQ_EMPTY) { if (np || len) return false; continue; }
         if (state != AVMP_REQ_LIVE && state != AVMP_REQ_KV_ONLY) return false;
-        if (np > g.max_pages || ((uint64_t)len + g.T - 1) / g.T != np) return false;
+        // a held request has at least one token (ADMIT and EXTEND reject zero tokens)
+        if (len == 0 || np > g.max_pages || ((uint64_t)len + g.T - 1) / g.T != np) return false;
         for (uint32_t j = 0; j < np; ++j) {
             const uint32_t h = t->req_chain[(size_t)r * g.max_pages + j], v = h & 0x7FFFFFFFu;
             if ((h >> 31) != AVMP_POOL_KV || v >= g.V[0] || t->vt[0][v] == kInvalid || ref[0][v]) return false;

@@ -88,3 +88,74 @@ class PayloadHarness:
             assert bad == 0
             assert np.array_equal(st, es) and np.array_equal(cv, ec)
         return total
+
+
+LAYOUT_SHAPES = [
+    W.ModelShape(3, 2, 4, 2, 4, 2, 64, 16, 4),   # rows, state and window are 16-byte multiples
+    W.ModelShape(2, 3, 4, 1, 3, 2, 5, 2, 4),     # 6-byte rows, 20 + 8 byte blocks padded to 32
+]
+
+
+def layout_workload(shape: W.ModelShape) -> W.Workload:
+    """Room for 16 pages and 16 blocks, 8 request slots, a migration allowed at every operation: random
+    batches followed by pure growth make both stores cede space that holds live units."""
+    u_kv = shape.n_attn_layers * 2 * shape.page_tokens * shape.kv_row_bytes
+    u_ssm = (shape.state_bytes + shape.conv_bytes + 15) // 16 * 16
+    pool = (16 * u_kv + 16 * u_ssm + 127) // 128 * 128
+    return W.Workload("layout", shape, pool, 16 * u_ssm / pool, 5, 8, 8, 12, "queue", 0, min_rebalance_interval_ops=1)
+
+
+def check_unit_layout(w: W.Workload, engine, read_units, rounds: int = 12, seed: int = 5) -> dict:
+    """Where inside a unit every byte lives, checked on the RAW bytes of the stores.
+
+    The contract (include/avmp.h, model shape): a KV page is the array
+    [attention layer][K, V][token in page][head][dim] of kv_elem_bytes elements; an SSM block is
+    the state elements followed by the convolution window.  Known rows go in through the engine's
+    scatter; a batch of pure growth then forces migrations that relocate some of the units just
+    written; the bytes are then read back NOT through a gather but from the unit's address
+    (`read_units(pool, handles) -> uint8[n][unit_bytes]`, which resolves the handles with
+    translate and reads the store itself) and compared through a numpy reshape of the unit to the
+    array shape above.  `engine` has step / scatter_kv / scatter_ssm / tables / stats."""
+    m = w.model
+    T, row, na = m.page_tokens, m.kv_row_bytes, m.n_attn_layers
+    R, MP = w.max_requests, w.max_pages
+    rng = np.random.default_rng(seed)
+    seen = dict(kv_rows=0, ssm_blocks=0)
+    for rnd in range(rounds):
+        engine.step(W.random_op_string(seed * 1000 + rnd, 24, R, T * 3, p_invalid=0.0))
+        t = engine.tables()
+        held = np.flatnonzero(t["req_state"] != 0).astype(np.uint32)
+        live = np.flatnonzero(t["req_state"] == 1).astype(np.uint32)
+        lens = t["req_len"][held].astype(np.int64)
+        tot = int(lens.sum())
+        kb = rng.integers(0, 256, (na, 2, tot, row), dtype=np.uint8)
+        for layer in range(na):
+            assert engine.scatter_kv(layer, held, np.zeros(len(held), np.uint32), kb[layer, 0], kb[layer, 1]) == 0
+        sb = rng.integers(0, 256, (m.n_ssm_layers, len(live), m.state_bytes), dtype=np.uint8)
+        cb = rng.integers(0, 256, (m.n_ssm_layers, len(live), m.conv_bytes), dtype=np.uint8)
+        for layer in range(m.n_ssm_layers):
+            assert engine.scatter_ssm(layer, live, sb[layer], cb[layer]) == 0
+        engine.step(W.make_ops(W.OP_EXTEND, live, T + 1))          # growth: migrations move written units
+        t = engine.tables()
+        chain = t["req_chain"].reshape(R, MP)
+        src = np.concatenate([[0], np.cumsum(lens)])
+        for k, r in enumerate(held):
+            n_old = int(lens[k])
+            pages = read_units(0, chain[r, : -(-n_old // T)])
+            for j, unit in enumerate(pages):
+                page = unit[: na * 2 * T * row].reshape(na, 2, T, row)   # [layer][K, V][token][head x dim]
+                n_tok = min(T, n_old - j * T)
+                want = kb[:, :, src[k] + j * T: src[k] + j * T + n_tok]
+                assert np.array_equal(page[:, :, :n_tok], want), f"round {rnd}: page {j} of request {r}"
+                seen["kv_rows"] += n_tok * na * 2
+        ssm = t["req_ssm"].reshape(R, m.n_ssm_layers)
+        for k, r in enumerate(live):
+            if t["req_state"][r] != 1:
+                continue
+            blocks = read_units(1, ssm[r])
+            for layer, unit in enumerate(blocks):
+                assert np.array_equal(unit[: m.state_bytes], sb[layer, k]), f"round {rnd}: state of request {r}"
+                assert np.array_equal(unit[m.state_bytes: m.state_bytes + m.conv_bytes], cb[layer, k])
+                seen["ssm_blocks"] += 1
+    seen["relocated_blocks"] = engine.stats()["relocated_blocks"]
+    return seen

@@ -40,6 +40,7 @@ def check_invariants(stats: dict, t: dict, *, page_tokens: int, n_ssm_layers: in
     ssm = t["req_ssm"].reshape(R, max(n_ssm_layers, 1))[:, :n_ssm_layers] if n_ssm_layers else None
     holds = st != EMPTY
     assert (npg[~holds] == 0).all() and (ln[~holds] == 0).all()
+    assert (ln[holds] >= 1).all()          # a held request has at least one token: zero-token ops are rejected
     assert (npg == -(-ln.astype(np.int64) // page_tokens)).all()
     kv_handles = np.concatenate([chain[r, :npg[r]] for r in np.flatnonzero(holds)] or [np.zeros(0, np.uint32)])
     assert len(kv_handles) == used_units[0]

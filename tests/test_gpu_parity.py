@@ -885,3 +885,60 @@ def test_import_rejects_inconsistent_snapshots(env):
     env["same"](g, o, w, "after importing the good snapshot")
     ops = d.next_batch()
     assert np.array_equal(g.step(ops), o.step(ops))
+
+
+def test_import_rejects_a_held_request_without_tokens(env):
+    """ADMIT and EXTEND take at least one token, so no sequence of operations leaves a held request
+    with zero tokens; a snapshot that says otherwise (its page returned to the free lists by hand, every
+    other table consistent) is refused, so the gathers never meet a request without rows."""
+    from paper_2605_22416_b200.binding import AvmpError
+    w = W.config("tiny")
+    g, o = _pair(env, w)
+    ops = W.make_ops(W.OP_ADMIT, [0], 1)
+    assert np.array_equal(g.step(ops), o.step(ops))
+    t, s = g.ctx.export_tables()
+    g.ctx.import_tables(t, s)                                   # as exported: accepted
+    h = int(t["req_chain"][0])
+    slot = int(t["vt_kv"][h])
+    t["slot_stack_kv"] = np.append(t["slot_stack_kv"], np.uint32(slot))
+    t["vid_stack_kv"] = np.append(t["vid_stack_kv"], np.uint32(h))
+    t["vt_kv"][h] = 0xFFFFFFFF
+    t["ow_kv"][slot] = 0xFFFFFFFF
+    t["req_len"][0] = 0
+    t["req_npages"][0] = 0
+    s["free_kv"] += 1
+    with pytest.raises(AvmpError):
+        g.ctx.import_tables(t, s)
+    env["same"](g, o, w, "context untouched")
+
+
+@pytest.mark.parametrize("shape", range(2))
+def test_bytes_inside_a_unit_follow_the_documented_layout_on_gpu(env, shape):
+    """The same raw-byte check as the oracle's pin, on the device arena: handles resolved with
+    avmp_translate (d_arena_offset), the unit read straight from the arena tensor and viewed as
+    [layer][K, V][token][head][dim] (state then window for SSM blocks), after migrations have
+    relocated some of the written units.  Shape 0 takes the bulk-copy kernels, shape 1 the generic ones."""
+    from harness import LAYOUT_SHAPES, check_unit_layout, layout_workload
+    w = layout_workload(LAYOUT_SHAPES[shape])
+    g = env["GpuEngine"](w)
+    s = g.stats()
+    unit = (s["unit_bytes_kv"], s["unit_bytes_ssm"])
+    arena = g.ctx.arena
+
+    def read_units(pool, handles):
+        p, off, bad, aoff = g.translate(np.asarray(handles, np.uint32))
+        assert bad == 0 and (p == pool).all()
+        return [arena[int(a): int(a) + unit[pool]].cpu().numpy() for a in aoff]
+
+    seen = check_unit_layout(w, g, read_units)
+    assert seen["kv_rows"] > 1000 and seen["ssm_blocks"] > 40 and seen["relocated_blocks"] > 4
+    assert g.stats()["error_code"] == 0
+    # and the same bytes through the oracle's stores: both sides place every byte alike
+    o = env["Oracle"].from_workload(w, with_store=True)
+
+    def read_units_o(pool, handles):
+        p, off, bad = o.translate(np.asarray(handles, np.uint32))
+        return [o.store_bytes(pool, int(x), unit[pool]) for x in off]
+
+    assert check_unit_layout(w, o, read_units_o) == seen
+    env["same"](g, o, w, "layout run")

@@ -541,3 +541,26 @@ def test_invalid_ops_advance_the_clock_and_change_nothing():
     t1, t2 = o.tables(), o2.tables()
     assert all(np.array_equal(t1[k], t2[k]) for k in t1)
     assert before != ""
+
+
+# ---- bytes inside a unit (Section 3.1 unit contents; layout promised by the C header) ---------
+from harness import LAYOUT_SHAPES, check_unit_layout, layout_workload  # noqa: E402
+
+
+@pytest.mark.parametrize("shape", LAYOUT_SHAPES)
+def test_bytes_inside_a_unit_follow_the_documented_layout(shape):
+    """A KV page is [layer][K, V][token][head][dim], an SSM block is state then window: read from the
+    raw store bytes at the translated offsets, after migrations have relocated written units."""
+    w = layout_workload(shape)
+    o = Oracle.from_workload(w, with_store=True)
+    s = o.stats()
+    unit = (s["unit_bytes_kv"], s["unit_bytes_ssm"])
+
+    def read_units(pool, handles):
+        p, off, bad = o.translate(np.asarray(handles, np.uint32))
+        assert bad == 0 and (p == pool).all()
+        return [o.store_bytes(pool, int(x), unit[pool]) for x in off]
+
+    seen = check_unit_layout(w, o, read_units)
+    assert seen["kv_rows"] > 1000 and seen["ssm_blocks"] > 40 and seen["relocated_blocks"] > 4
+    _inv(o, w)
