@@ -6,12 +6,16 @@ avmp_step (admit / extend / finish batch, CapacityError handler, migration + rel
 copy), avmp_translate of every live handle of the running batch, avmp_gather_kv for every
 attention layer and avmp_gather_ssm for every SSM layer of the running batch.
 
-Workload: the short-uniform mix (Jamba-like 4 attention + 28 Mamba layers, 4 GiB pool,
-split 0.5, B = 128, step batch 256), synthetic and seeded.  The trace is produced closed
-loop against the library itself (untimed), then replayed from device-resident op batches
-for the timed region.  Inputs exceed L2: every step reads and writes several GB.
+Workload of the headline: `scale`, the largest single-GPU configuration (72-layer hybrid, 9
+attention + 63 Mamba layers, 120 GiB pool resident in HBM, split 0.5, B = 128, step batch
+1024), synthetic and seeded.  The trace is produced closed loop against the library itself
+(untimed), then replayed from device-resident op batches for the timed region.  Inputs exceed
+L2: every step reads and writes about 190 GB.  The other four configurations are measured
+the same way, briefly, and reported under roofline.other_configs.
 
-Prints ONE JSON line: headline value, roofline of the dominant kernel, end-to-end figure, CPU baseline.
+Prints ONE JSON line: headline value, roofline of the dominant kernel (with the secondary
+figures of the metric: KV gather, relocation copy, single-layer launches, allocator rate),
+end-to-end figure, CPU baseline.
 """
 from __future__ import annotations
 
@@ -32,11 +36,13 @@ from paper_2605_22416_b200 import workloads as W  # noqa: E402
 
 METRIC = "paged gather+migration GB/s over whole engine steps (allocator ops/s reported beside it)"
 WARM_STEPS = 600          # closed-loop steps before the measured window (steady state)
-# DRAM bytes (read + write) per launch of the dominant kernel divided by its algorithmic bytes, from an ncu
-# capture of this benchmark's own launches (profiles/bench_short_uniform_dram_traffic.md; the two byte counters
-# take one pass, so the full-size launches can be captured).  Reads equal the algorithmic bytes; the last
-# 0.7 % of the writes is still in L2 when the kernel ends.  A 1 GB launch of the same kernel reads 0.953.
-NCU_TRAFFIC_RATIO = 0.993
+# DRAM traffic of one launch of the dominant kernel, from ncu captures of this kernel (profiles/
+# ssm_gather_fused_jamba_like.md at 1 GB per launch, profiles/bench_short_uniform_dram_traffic.md at 6.8 GB):
+# reads equal the algorithmic read bytes, and of the writes about 47 MB are still dirty in L2 when the kernel
+# ends (they reach DRAM during the next kernel).  Recorded from those captures, not re-measured per run.
+L2_DIRTY_TAIL_BYTES = 47e6
+# timed steps and warm steps of the brief runs of the other configurations: each timed region exceeds 0.2 s
+OTHER_CONFIGS = {"pr1": (2600, 400), "short_uniform": (200, 600), "mixed_long": (420, 600), "agentic_burst": (130, 600)}
 
 
 def _peaks():
@@ -103,13 +109,18 @@ def step_bytes(model: W.ModelShape, n_running: int, total_tokens: int, relocated
 
 
 def config_dict(w: W.Workload, warm_steps: int = WARM_STEPS) -> dict:
+    """What the workload is (the same dict for both arms; what a run saw goes under `workload_stats`)."""
     m = w.model
     return {"workload": w.name, "cache_shape": f"{m.n_attn_layers} attention + {m.n_ssm_layers} mamba layers, "
                                                f"KV page {m.page_tokens} tok x {m.kv_heads} x {m.head_dim} bf16, "
                                                f"SSM block {m.ssm_state_elems} + {m.ssm_conv_elems} fp32",
             "pool_gib": w.pool_bytes / W.GiB,
             "split": w.split, "migration_batch_size": w.migration_batch_size, "step_batch": w.concurrency,
-            "warm_steps": warm_steps}
+            "warm_steps": warm_steps, "seed": w.seed,
+            "l2": "inputs larger than L2: every launch reads its bytes from a multi-GiB arena for the first time in "
+                  "the step and writes a batch buffer that the next group or step overwrites only after far more "
+                  "than L2's 126 MB has passed through",
+            "multi_gpu": "replicas only: one independent context per GPU, no collective"}
 
 
 def reduce_over_ranks(local_ms: float, local_sums: np.ndarray, world: int):
@@ -126,25 +137,41 @@ def reduce_over_ranks(local_ms: float, local_sums: np.ndarray, world: int):
     return float(t.item()), s.cpu().numpy()
 
 
+def layers_per_launch(w: W.Workload, dev, max_run: int, max_tok: int, asked: int):
+    """How many layers of batch buffers fit beside the arena: all attention layers, and as many SSM layers
+    as the free memory holds (the launches of a step then walk the layers in groups of that size)."""
+    import torch
+    m = w.model
+    if asked:
+        return min(m.n_attn_layers, asked), min(m.n_ssm_layers, asked)
+    free, _ = torch.cuda.mem_get_info(dev)
+    free -= 6 * W.GiB                                            # tables, traces, slack
+    kv_layer = 2 * max_tok * m.kv_row_bytes
+    lpl_kv = int(max(1, min(m.n_attn_layers, (free // 2) // max(kv_layer, 1))))
+    free -= lpl_kv * kv_layer
+    ssm_layer = max_run * (m.state_bytes + m.conv_bytes)
+    lpl_ssm = int(max(1, min(m.n_ssm_layers, free // max(ssm_layer, 1))))
+    return lpl_kv, lpl_ssm
+
+
 # ---------------------------------------------------------------------------------------
 # our arm
 # ---------------------------------------------------------------------------------------
-def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
+def measure(w: W.Workload, dev, *, steps: int, warmup: int, warm_steps: int, asked_lpl: int, full: bool,
+            world: int = 1) -> dict:
+    """The hot path on one workload: K whole engine steps under one event pair, then the same window with an
+    event pair per kernel class.  full: also one launch per layer, and the end-to-end loop with host buffers."""
     import torch
     from paper_2605_22416_b200 import binding as B
 
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    w = W.config(args.workload, seed=rank % 3 if world > 1 else args.seed)
     m = w.model
-    WS = args.warm_steps
-    n_steps = WS + args.warmup + args.steps
-    lpl_kv = min(m.n_attn_layers, args.layers_per_launch or m.n_attn_layers)
-    lpl_ssm = min(m.n_ssm_layers, args.layers_per_launch or m.n_ssm_layers)
+    WS = warm_steps
+    n_steps = WS + warmup + steps
 
     # ---- phase A: closed loop against the library (untimed) -> per-step batches ----
     ctx = B.Context.from_workload(w, device=dev)
-    drv = W.ClosedLoopDriver(w)
+    drv = W.ClosedLoopDriver(w, requests=W.make_requests(w, min(w.n_requests, 400 * w.concurrency))
+                             if w.kind == "queue" else None)
     trace = []
 
     def held_units():
@@ -169,7 +196,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
             rec["handles"] = np.concatenate([chain[r, :t["req_npages"][r]] for r in rec["run"]] +
                                             [ssm[rec["run"]].reshape(-1)]).astype(np.uint32)
         trace.append(rec)
-    assert len(trace) == n_steps, "trace ended before the measured window"
+    assert len(trace) == n_steps, f"{w.name}: trace ended after {len(trace)} of {n_steps} steps"
     stats_a = ctx.stats()
     arena = ctx.arena
     ctx.close()
@@ -177,11 +204,13 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     # ---- phase B: replay from device-resident batches ----
     stream = torch.cuda.current_stream()
     sid = stream.cuda_stream          # raw cudaStream_t, passed straight to the C ABI
-    max_run = max(len(r["run"]) for r in trace[WS:])
-    max_tok = max(int(r["lens"].sum()) for r in trace[WS:])
-    max_h = max(len(r["handles"]) for r in trace[WS:])
+    max_run = max(max(len(r["run"]) for r in trace[WS:]), 1)
+    max_tok = max(max(int(r["lens"].sum()) for r in trace[WS:]), 1)
+    max_h = max(max(len(r["handles"]) for r in trace[WS:]), 1)
+    lpl_kv, lpl_ssm = layers_per_launch(w, dev, max_run, max_tok, asked_lpl)
     d_status = torch.zeros(w.concurrency * 2 + 16, dtype=torch.int32, device=dev)
-    # batch buffers: one slab per kind, [layer][row]; every layer has its own rows (no buffer reuse)
+    # batch buffers: one slab per kind, [layer][row]; the layers of a launch have their own rows (no reuse
+    # inside a launch; the next group of layers reuses the slab)
     out_k = torch.empty((lpl_kv, max_tok, m.kv_row_bytes), dtype=torch.uint8, device=dev)
     out_v = torch.empty((lpl_kv, max_tok, m.kv_row_bytes), dtype=torch.uint8, device=dev)
     out_s = torch.empty((lpl_ssm, max_run, m.state_bytes), dtype=torch.uint8, device=dev)
@@ -207,25 +236,16 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     def ev():
         return torch.cuda.Event(enable_timing=True)
 
-    def fresh_context(full_warmup=True):
-        """A new context over the same arena, replayed up to the start of the timed window."""
-        c = B.Context.from_workload(w, device=dev, arena=arena)
-        for r in trace[:WS]:
-            c.step(r["d_ops"], len(r["ops"]), d_status, sid)
-        for r in trace[WS:WS + args.warmup]:
-            if full_warmup:
-                full_step(c, r)
-            else:
-                c.step(r["d_ops"], len(r["ops"]), d_status, sid)
-        torch.cuda.synchronize(dev)
-        return c
+    # when the batch buffers of all layers fit, a step's payload moves in ONE launch (avmp_gather_step)
+    one_launch = len(kv_groups) == 1 and len(ssm_groups) == 1
 
-    def full_step(c, r, marks=None, per_layer=False, d_run=None):
+    def full_step(c, r, marks=None, per_layer=False, fused=False):
         """One engine step.  marks: one event pair per kernel class (allocator, KV, SSM).
-        per_layer: one launch per layer instead of one launch for all layers."""
+        per_layer: one launch per layer instead of one launch per group of layers.
+        fused: both gathers of all layers in one launch (the KV mark then coincides with the allocator mark)."""
         n_ops, n_run = len(r["ops"]), len(r["run"])
         cap_tok = int(r["lens"].sum())
-        run = r["d_run"] if d_run is None else d_run
+        run = r["d_run"]
         e = [ev() for _ in range(4)] if marks is not None else None
         if e:
             e[0].record(stream)
@@ -233,6 +253,14 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
         c.translate(r["d_handles"], len(r["handles"]), d_pool, d_off, d_aoff, sid)
         if e:
             e[1].record(stream)
+        if fused:
+            c.gather_step(run, n_run, 0, m.n_attn_layers, out_k, out_v, kv_stride, cap_tok, d_cu,
+                          0, m.n_ssm_layers, out_s, s_stride, out_c, c_stride, sid)
+            if e:
+                e[2].record(stream)
+                e[3].record(stream)
+                marks.append(e)
+            return
         if per_layer:
             for l in range(m.n_attn_layers):
                 c.gather_kv(l, run, n_run, out_k[l % lpl_kv], out_v[l % lpl_kv], cap_tok, d_cu, sid)
@@ -251,7 +279,20 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
             e[3].record(stream)
             marks.append(e)
 
-    timed = trace[WS + args.warmup:]
+    def fresh_context(full_warmup=True):
+        """A new context over the same arena, replayed up to the start of the timed window."""
+        c = B.Context.from_workload(w, device=dev, arena=arena)
+        for r in trace[:WS]:
+            c.step(r["d_ops"], len(r["ops"]), d_status, sid)
+        for r in trace[WS:WS + warmup]:
+            if full_warmup:
+                full_step(c, r, fused=one_launch)
+            else:
+                c.step(r["d_ops"], len(r["ops"]), d_status, sid)
+        torch.cuda.synchronize(dev)
+        return c
+
+    timed = trace[WS + warmup:]
 
     # ---- timed region 1: K whole steps, one pair of events, nothing else on the stream ----
     ctx = fresh_context()
@@ -260,13 +301,13 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
         import torch.distributed as dist
         dist.barrier()
     torch.cuda.synchronize(dev)
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(dev.index or 0)
     sampler.start()
     launches0 = ctx.launch_count()
     e0, e1 = ev(), ev()
     e0.record(stream)
     for r in timed:
-        full_step(ctx, r)
+        full_step(ctx, r, fused=one_launch)
     e1.record(stream)
     torch.cuda.synchronize(dev)
     if world > 1:
@@ -278,11 +319,11 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     ctx.close()
 
     # ---- region 2: the same window again with one event pair per kernel class and step ----
-    def timed_classes(per_layer):
+    def timed_classes(per_layer, fused=False):
         c = fresh_context()
         marks = []
         for r in timed:
-            full_step(c, r, marks, per_layer=per_layer)
+            full_step(c, r, marks, per_layer=per_layer, fused=fused)
         torch.cuda.synchronize(dev)
         st = c.stats()
         c.close()
@@ -293,97 +334,176 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
                  "ssm": [e[2].elapsed_time(e[3]) / nl_ssm for e in marks]}, st)
 
     per, st_c = timed_classes(per_layer=False)
-    per_l, _ = timed_classes(per_layer=True)
+    per_l = timed_classes(per_layer=True)[0] if full else None
+    per_f = timed_classes(per_layer=False, fused=True)[0] if one_launch else None
     clocks = sampler.stop()
 
     # ---- e2e: host buffers in, host results out, every step ----
-    ctx = fresh_context(full_warmup=False)
-    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.uint8).reshape(-1).copy()).pin_memory()
-    h_ops = [pin(r["ops"]) if len(r["ops"]) else torch.zeros(16, dtype=torch.uint8).pin_memory() for r in timed]
-    h_run = [pin(r["run"]) for r in timed]
-    h_status = torch.zeros(w.concurrency * 2 + 16, dtype=torch.int32).pin_memory()
-    h_cu = torch.zeros(max_run + 1, dtype=torch.int32).pin_memory()
-    d_run_buf = torch.zeros(max_run * 4 + 16, dtype=torch.uint8, device=dev)
-    h2d = d2h = 0
-    torch.cuda.synchronize(dev)
-    t0 = time.perf_counter()
-    for r, ho, hr in zip(timed, h_ops, h_run):
-        n_ops, n_run = len(r["ops"]), len(r["run"])
-        ctx.step_host(ho, n_ops, h_status, sid)                    # H2D ops, D2H statuses, sync
-        d_run_buf[: hr.numel()].copy_(hr, non_blocking=True)       # H2D running list
-        cap_tok = int(r["lens"].sum())
-        for f, nl in kv_groups:
-            ctx.gather_kv_layers(f, nl, d_run_buf, n_run, out_k, out_v, kv_stride, cap_tok, d_cu, sid)
-        for f, nl in ssm_groups:
-            ctx.gather_ssm_layers(f, nl, d_run_buf, n_run, out_s, s_stride, out_c, c_stride, sid)
-        h_cu[: n_run + 1].copy_(d_cu[: n_run + 1], non_blocking=True)   # D2H row offsets of the batch
+    e2e_ms, h2d, d2h = None, 0, 0
+    if full:
+        ctx = fresh_context(full_warmup=False)
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.uint8).reshape(-1).copy()).pin_memory()
+        h_ops = [pin(r["ops"]) if len(r["ops"]) else torch.zeros(16, dtype=torch.uint8).pin_memory() for r in timed]
+        h_run = [pin(r["run"]) if len(r["run"]) else torch.zeros(16, dtype=torch.uint8).pin_memory() for r in timed]
+        h_status = torch.zeros(w.concurrency * 2 + 16, dtype=torch.int32).pin_memory()
+        h_cu = torch.zeros(max_run + 1, dtype=torch.int32).pin_memory()
+        d_run_buf = torch.zeros(max_run * 4 + 16, dtype=torch.uint8, device=dev)
         torch.cuda.synchronize(dev)
-        h2d += n_ops * 12 + n_run * 4
-        d2h += n_ops * 4 + (n_run + 1) * 4
-    e2e_ms = (time.perf_counter() - t0) * 1e3
-    ctx.close()
+        t0 = time.perf_counter()
+        for r, ho, hr in zip(timed, h_ops, h_run):
+            n_ops, n_run = len(r["ops"]), len(r["run"])
+            ctx.step_host(ho, n_ops, h_status, sid)                    # H2D ops, D2H statuses, sync
+            d_run_buf[: n_run * 4].copy_(hr[: n_run * 4], non_blocking=True)   # H2D running list
+            cap_tok = int(r["lens"].sum())
+            if one_launch:
+                ctx.gather_step(d_run_buf, n_run, 0, m.n_attn_layers, out_k, out_v, kv_stride, cap_tok, d_cu,
+                                0, m.n_ssm_layers, out_s, s_stride, out_c, c_stride, sid)
+            else:
+                for f, nl in kv_groups:
+                    ctx.gather_kv_layers(f, nl, d_run_buf, n_run, out_k, out_v, kv_stride, cap_tok, d_cu, sid)
+                for f, nl in ssm_groups:
+                    ctx.gather_ssm_layers(f, nl, d_run_buf, n_run, out_s, s_stride, out_c, c_stride, sid)
+            h_cu[: n_run + 1].copy_(d_cu[: n_run + 1], non_blocking=True)   # D2H row offsets of the batch
+            torch.cuda.synchronize(dev)
+            h2d += n_ops * 12 + n_run * 4
+            d2h += n_ops * 4 + (n_run + 1) * 4
+        e2e_ms = (time.perf_counter() - t0) * 1e3
+        ctx.close()
 
     # ---- accounting ----
     K = len(timed)
     by = [step_bytes(m, len(r["run"]), int(r["lens"].sum()), 0) for r in timed]
     kv_bytes = sum(b["kv"] for b in by)
     ssm_bytes = sum(b["ssm"] for b in by)
-    moved = kv_bytes + ssm_bytes + 2 * reloc_timed
-    n_ops_total = sum(len(r["ops"]) for r in timed)
-    local_sums = np.array([moved, n_ops_total, kv_bytes, ssm_bytes, launches, h2d, d2h], dtype=np.float64)
-    total_ms_g, sums = reduce_over_ranks(total_ms, local_sums, world)
-    e2e_ms_g, _ = reduce_over_ranks(e2e_ms, np.zeros(1), world)
-    peak, peak_kind = _peaks()
+    res = {
+        "K": K, "total_ms": total_ms, "e2e_ms": e2e_ms, "h2d": h2d, "d2h": d2h, "launches": launches,
+        "kv_bytes": kv_bytes, "ssm_bytes": ssm_bytes, "reloc_bytes": reloc_timed,
+        "moved": kv_bytes + ssm_bytes + 2 * reloc_timed,
+        "n_ops": sum(len(r["ops"]) for r in timed), "units": sum(r["units"] for r in timed),
+        "per": per, "per_l": per_l, "per_f": per_f, "one_launch": one_launch, "clocks": clocks, "lpl": (lpl_kv, lpl_ssm),
+        "n_kv_launches": len(kv_groups), "n_ssm_launches": len(ssm_groups),
+        "running_mean": float(np.mean([len(r["run"]) for r in timed])),
+        "tokens_mean": float(np.mean([int(r["lens"].sum()) for r in timed])),
+        "rebalances": st_c["n_rebalance"], "n_oom": st_c["n_oom"],
+        "replay_matches": all(st_b[k] == stats_a[k] for k in stats_a if not k.startswith(("relocation_ns", "step_ns"))),
+    }
+    del out_k, out_v, out_s, out_c, arena, trace, timed
+    torch.cuda.empty_cache()
+    return res
 
-    ssm_launch_bytes = ssm_bytes / (K * len(ssm_groups))   # by default one launch gathers all SSM layers of a step
-    ssm_avg_ms = float(np.mean(per["ssm"]))
-    achieved = ssm_launch_bytes / (ssm_avg_ms * 1e-3) / 1e9
-    kv_launch_bytes = kv_bytes / (K * len(kv_groups))
-    kv_avg_ms = float(np.mean(per["kv"]))
-    step_avg_ms = float(np.mean(per["step"]))
-    pl_ssm = (ssm_bytes / (K * m.n_ssm_layers)) / (float(np.mean(per_l["ssm"])) * 1e-3) / 1e9
-    pl_kv = (kv_bytes / (K * m.n_attn_layers)) / (float(np.mean(per_l["kv"])) * 1e-3) / 1e9
+
+def class_figures(res: dict, m: W.ModelShape, peak: float) -> dict:
+    """GB/s and fractions of the copy-kernel classes of one measured workload, from bytes by definition of the
+    operations and event-timed launch durations."""
+    K = res["K"]
+    per = res["per"]
+    ssm_launch_bytes = res["ssm_bytes"] / (K * res["n_ssm_launches"])
+    kv_launch_bytes = res["kv_bytes"] / (K * res["n_kv_launches"])
+    ssm_ms, kv_ms, step_ms = float(np.mean(per["ssm"])), float(np.mean(per["kv"])), float(np.mean(per["step"]))
+    out = {"ssm_gbs": ssm_launch_bytes / (ssm_ms * 1e-3) / 1e9, "ssm_launch_ms": ssm_ms, "ssm_launch_bytes": ssm_launch_bytes,
+           "kv_gbs": kv_launch_bytes / (kv_ms * 1e-3) / 1e9, "kv_launch_ms": kv_ms, "kv_launch_bytes": kv_launch_bytes,
+           "allocator_us_per_step": step_ms * 1e3, "allocator_ops_per_s": res["n_ops"] / (sum(per["step"]) * 1e-3),
+           "unit_allocs_frees_per_s": res["units"] / (sum(per["step"]) * 1e-3)}
+    if res["per_f"] is not None:
+        ms = float(np.mean([a + b for a, b in zip(res["per_f"]["kv"], res["per_f"]["ssm"])]))   # kv mark is empty
+        out["step_gather_gbs"] = (res["kv_bytes"] + res["ssm_bytes"]) / K / (ms * 1e-3) / 1e9
+        out["step_gather_launch_ms"] = ms
+    if res["per_l"] is not None:
+        pl = res["per_l"]
+        out["single_layer_ssm_gbs"] = (res["ssm_bytes"] / (K * m.n_ssm_layers)) / (float(np.mean(pl["ssm"])) * 1e-3) / 1e9
+        out["single_layer_kv_gbs"] = (res["kv_bytes"] / (K * m.n_attn_layers)) / (float(np.mean(pl["kv"])) * 1e-3) / 1e9
+        out["single_layer_ssm_launch_ms"] = float(np.mean(pl["ssm"]))
+        out["single_layer_kv_launch_ms"] = float(np.mean(pl["kv"]))
+    return out
+
+
+def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
+    import torch
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    w = W.config(args.workload, seed=rank % 3 if world > 1 else args.seed)
+    m = w.model
+    peak, peak_kind = _peaks()
+    res = measure(w, dev, steps=args.steps, warmup=args.warmup, warm_steps=args.warm_steps,
+                  asked_lpl=args.layers_per_launch, full=True, world=world)
+    K = res["K"]
+    local_sums = np.array([res["moved"], res["n_ops"], res["kv_bytes"], res["ssm_bytes"], res["launches"],
+                           res["h2d"], res["d2h"]], dtype=np.float64)
+    total_ms_g, sums = reduce_over_ranks(res["total_ms"], local_sums, world)
+    e2e_ms_g, _ = reduce_over_ranks(res["e2e_ms"], np.zeros(1), world)
+    f = class_figures(res, m, peak)
+    lpl_kv, lpl_ssm = res["lpl"]
+    traffic = max(f["ssm_launch_bytes"] - L2_DIRTY_TAIL_BYTES, f["ssm_launch_bytes"] / 2)
     out = {
         "metric": METRIC, "value": sums[0] / (total_ms_g * 1e-3) / 1e9, "unit": "GB/s",
         "n_gpus": world, "steps": K, "warmup": args.warmup, "ms_per_step": total_ms_g / K,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u32",
         "data": "synthetic", "impl": "ours",
-        "config": {**config_dict(w, WS), "running_mean": float(np.mean([len(r["run"]) for r in timed])),
-                   "tokens_mean": float(np.mean([int(r["lens"].sum()) for r in timed])),
-                   "layers_per_launch": {"kv": lpl_kv, "ssm": lpl_ssm},
-                   "l2": "inputs larger than L2: every launch reads its bytes from a multi-GiB arena for the first time in the step and writes a batch buffer that the next group or step overwrites only after far more than L2's 126 MB has passed through",
-                   "multi_gpu": "replicas only: one independent context per GPU, no collective"},
-        "allocator": {"ops_per_s": sums[1] / (sum(per["step"]) * 1e-3) * (world if world > 1 else 1),
-                      "us_per_step": step_avg_ms * 1e3, "ops_per_step": n_ops_total / K,
-                      "units_per_step": sum(r["units"] for r in timed) / K,
-                      "unit_allocs_and_frees_per_s": sum(r["units"] for r in timed) / (sum(per["step"]) * 1e-3),
-                      "note": "avmp_step + avmp_translate, CUDA events around the two calls, rank 0's timing; units = "
-                              "KV pages + SSM blocks allocated or freed, counted from the request slots' net change per step"},
-        "gather_kv": {"gbs": kv_launch_bytes / (kv_avg_ms * 1e-3) / 1e9, "avg_launch_ms": kv_avg_ms,
-                      "frac_of_peak": kv_launch_bytes / (kv_avg_ms * 1e-3) / 1e9 / peak,
-                      "note": "avmp_gather_kv_layers: one copy launch for all attention layers (the request-list plan is computed inside it)"},
-        "per_layer_launches": {"gather_ssm_gbs": pl_ssm, "gather_ssm_frac_of_peak": pl_ssm / peak,
-                               "gather_ssm_avg_launch_ms": float(np.mean(per_l["ssm"])),
-                               "gather_kv_gbs": pl_kv, "gather_kv_frac_of_peak": pl_kv / peak,
-                               "note": "same window with avmp_gather_ssm / avmp_gather_kv called once per layer"},
-        "migration": {"relocated_bytes_in_window": int(reloc_timed), "rebalances_total": st_c["n_rebalance"],
-                      "n_oom_total": st_c["n_oom"]},
-        "roofline": {"kernel": f"stream_bulk_kernel<SsmPieces<gather>> (avmp_gather_ssm_layers, {lpl_ssm} SSM layers per launch)", "bound": "hbm", "achieved": achieved, "peak": peak,
-                     "unit": "GB/s", "frac": achieved / peak, "peak_source": f"MEASURED_PEAKS.json hbm_gbs ({peak_kind})",
-                     "frac_of_nominal_8000": achieved / 8000.0, "avg_launch_ms": ssm_avg_ms,
-                     "bytes_per_launch": ssm_launch_bytes,
-                     "traffic": None if NCU_TRAFFIC_RATIO is None else ssm_launch_bytes * NCU_TRAFFIC_RATIO},
+        "config": config_dict(w, args.warm_steps),
+        "workload_stats": {"running_mean": res["running_mean"], "tokens_mean": res["tokens_mean"],
+                           "ops_per_step": res["n_ops"] / K, "units_per_step": res["units"] / K,
+                           "layers_per_launch": {"kv": lpl_kv, "ssm": lpl_ssm},
+                           "relocated_bytes_in_window": int(res["reloc_bytes"]), "rebalances_total": res["rebalances"],
+                           "n_oom_total": res["n_oom"], "replay_matches_closed_loop": res["replay_matches"]},
+        "roofline": {"kernel": f"stream_bulk_kernel<SsmPieces<gather>> (avmp_gather_ssm_layers, {lpl_ssm} SSM layers per launch)",
+                     "bound": "hbm", "achieved": f["ssm_gbs"], "peak": peak, "unit": "GB/s", "frac": f["ssm_gbs"] / peak,
+                     "peak_source": f"MEASURED_PEAKS.json hbm_gbs ({peak_kind})",
+                     "frac_of_nominal_8000": f["ssm_gbs"] / 8000.0, "avg_launch_ms": f["ssm_launch_ms"],
+                     "bytes_per_launch": f["ssm_launch_bytes"], "traffic": traffic,
+                     "traffic_source": "algorithmic bytes minus the ~47 MB of output still dirty in L2 at kernel end "
+                                       "(ncu captures of this kernel at 1 GB and 6.8 GB per launch, profiles/); "
+                                       "recorded from those captures, not measured in this run",
+                     "secondary": {
+                         "kv_gather": {"gbs": f["kv_gbs"], "frac": f["kv_gbs"] / peak, "avg_launch_ms": f["kv_launch_ms"],
+                                       "bytes_per_launch": f["kv_launch_bytes"],
+                                       "note": f"avmp_gather_kv_layers, {lpl_kv} attention layers per launch, plan computed inside the launch"},
+                         "single_layer_ssm": {"gbs": f["single_layer_ssm_gbs"], "frac": f["single_layer_ssm_gbs"] / peak,
+                                              "avg_launch_ms": f["single_layer_ssm_launch_ms"],
+                                              "note": "same window, avmp_gather_ssm once per layer, back to back"},
+                         "single_layer_kv": {"gbs": f["single_layer_kv_gbs"], "frac": f["single_layer_kv_gbs"] / peak,
+                                             "avg_launch_ms": f["single_layer_kv_launch_ms"],
+                                             "note": "same window, avmp_gather_kv once per layer, back to back"},
+                         "allocator_ops_per_s": f["allocator_ops_per_s"] * (world if world > 1 else 1),
+                         "allocator_us_per_step": f["allocator_us_per_step"],
+                         "unit_allocs_frees_per_s": f["unit_allocs_frees_per_s"],
+                         "allocator_note": "avmp_step + avmp_translate of every live handle of the batch, CUDA events "
+                                           "around the two calls, rank 0's timing; units = KV pages + SSM blocks allocated "
+                                           "or freed, counted from the request slots' net change per step"}},
         "e2e": {"value": sums[0] / (e2e_ms_g * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms_g / K,
                 "h2d_bytes_per_step": sums[5] / K / world, "d2h_bytes_per_step": sums[6] / K / world,
                 "note": "ops and running list from pinned host memory, statuses and row offsets back to the host every step; gathered batch buffers stay in HBM for the model's kernels"},
         "gpu_launches": int(sums[4]),
-        "clocks": clocks,
+        "clocks": res["clocks"],
         "paper_context": "the paper (pure-Python prototype, one RTX 3060 12GB) reports 1.83-13.3x goodput and a 7.6 % "
                          "OOM reduction for dynamic rebalancing against its best static baseline; it reports no "
                          "allocator ops/s, GB/s or kernel timings, so vs_baseline is null",
-        "replay_matches_closed_loop": all(st_b[k] == stats_a[k] for k in stats_a if not k.startswith(("relocation_ns", "step_ns"))),
     }
     return out
+
+
+def other_configs(dev, skip: str) -> list:
+    """The other configurations, each measured briefly the same way (K whole steps under one event pair, then
+    per kernel class): whole-step GB/s and the fraction of the measured peak the two gathers reach."""
+    peak, _ = _peaks()
+    rows = []
+    for name, (k, ws) in OTHER_CONFIGS.items():
+        if name == skip:
+            continue
+        w = W.config(name)
+        res = measure(w, dev, steps=k, warmup=3, warm_steps=ws, asked_lpl=0, full=False)
+        f = class_figures(res, w.model, peak)
+        rows.append({"workload": name, "steps": res["K"], "timed_region_ms": res["total_ms"],
+                     "value": res["moved"] / (res["total_ms"] * 1e-3) / 1e9, "frac": res["moved"] / (res["total_ms"] * 1e-3) / 1e9 / peak,
+                     "ms_per_step": res["total_ms"] / res["K"],
+                     "running_mean": res["running_mean"], "tokens_mean": res["tokens_mean"],
+                     "ssm_gather_gbs": f["ssm_gbs"], "ssm_gather_frac": f["ssm_gbs"] / peak,
+                     "kv_gather_gbs": f["kv_gbs"], "kv_gather_frac": f["kv_gbs"] / peak,
+                     "step_gather_gbs": f.get("step_gather_gbs"),
+                     "step_gather_frac": f["step_gather_gbs"] / peak if "step_gather_gbs" in f else None,
+                     "gathers_per_step": "one launch (avmp_gather_step)" if res["one_launch"] else "one launch per kind and group of layers",
+                     "allocator_us_per_step": f["allocator_us_per_step"], "allocator_ops_per_s": f["allocator_ops_per_s"],
+                     "replay_matches_closed_loop": res["replay_matches"], "clocks": res["clocks"]})
+    return rows
 
 
 # ---------------------------------------------------------------------------------------
@@ -594,39 +714,57 @@ def allocator_scaling(dev, batches=(32, 256, 1024, 4096), warm=120, timed=60) ->
 # ---------------------------------------------------------------------------------------
 # the oracle on the host cores: cpu_baseline leg and the --impl reference arm
 # ---------------------------------------------------------------------------------------
-def run_oracle(args, n_sample_steps: int, budget_s: float = 25.0) -> dict:
+def run_oracle(args, n_sample_steps: int, budget_s: float = 25.0, warmup_steps: int = 0,
+               sample_bytes: float = 3.0e9) -> dict:
+    """The oracle as it stands, single thread, on a bounded sample of the same workload: every sampled step
+    runs the allocator update of the WHOLE batch, then translate and the all-layer gathers for the first
+    requests of the running batch whose units fit in `sample_bytes` of host memory (the oracle keeps real
+    stores; the whole batch of the large configurations would need more host memory than a box may have)."""
     from oracle.avmp_oracle import Oracle
     w = W.config(args.workload, seed=args.seed)
     m = w.model
     o = Oracle.from_workload(w, with_store=True)
-    drv = W.ClosedLoopDriver(w)
+    drv = W.ClosedLoopDriver(w, requests=W.make_requests(w, min(w.n_requests, 400 * w.concurrency))
+                             if w.kind == "queue" else None)
     while not drv.done and drv.step < args.warm_steps:
         ops = drv.next_batch()
         drv.feed(o.step(ops))
-    # give every live unit real bytes (the stores are committed lazily)
+
+    def sample_of(run, lens):
+        per_req = m.n_ssm_layers * (m.state_bytes + m.conv_bytes) + lens * 2 * m.kv_row_bytes * m.n_attn_layers
+        n = int(np.searchsorted(np.cumsum(per_req), sample_bytes, side="right"))
+        return max(1, min(n, len(run)))
+
+    # give every unit the sample can touch real bytes (the stores are committed lazily)
     run = drv.running_slots.astype(np.uint32)
+    ns0 = sample_of(run, drv.len[run]) if len(run) else 0
     rng = np.random.default_rng(0)
-    lens = drv.len[run]
-    for l in range(m.n_attn_layers):
-        kb = rng.integers(0, 256, (int(lens.sum()), m.kv_row_bytes), dtype=np.uint8)
-        o.scatter_kv(l, run, np.zeros(len(run), np.uint32), kb, kb)
-    sb = rng.integers(0, 256, (len(run), m.state_bytes), dtype=np.uint8)
-    cb = rng.integers(0, 256, (len(run), m.conv_bytes), dtype=np.uint8)
-    for l in range(m.n_ssm_layers):
-        o.scatter_ssm(l, run, sb, cb)
+    if ns0:
+        srun, slens = run[:ns0], drv.len[run[:ns0]]
+        kb = rng.integers(0, 256, (int(slens.sum()), m.kv_row_bytes), dtype=np.uint8)
+        for l in range(m.n_attn_layers):
+            o.scatter_kv(l, srun, np.zeros(ns0, np.uint32), kb, kb)
+        sb = rng.integers(0, 256, (ns0, m.state_bytes), dtype=np.uint8)
+        cb = rng.integers(0, 256, (ns0, m.conv_bytes), dtype=np.uint8)
+        for l in range(m.n_ssm_layers):
+            o.scatter_ssm(l, srun, sb, cb)
     moved = n_ops = 0
     t_alloc = t_total = 0.0
     steps = 0
-    while steps < n_sample_steps and t_total < budget_s and not drv.done:
+    sampled, batch = [], []
+    while steps < warmup_steps + n_sample_steps and t_total < budget_s and not drv.done:
         ops = drv.next_batch()
         t0 = time.perf_counter()
         st = o.step(ops)
         t1 = time.perf_counter()
         drv.feed(st)
         run = drv.running_slots.astype(np.uint32)
+        if len(run) == 0:
+            continue
+        ns = sample_of(run, drv.len[run])
+        run = run[:ns]
         lens = drv.len[run]
         tot = int(lens.sum())
-        t2 = time.perf_counter()
         tb = o.tables()
         chain = tb["req_chain"].reshape(w.max_requests, w.max_pages)
         handles = np.concatenate([chain[r, :tb["req_npages"][r]] for r in run] +
@@ -638,29 +776,37 @@ def run_oracle(args, n_sample_steps: int, budget_s: float = 25.0) -> dict:
         for l in range(m.n_ssm_layers):
             o.gather_ssm(l, run)
         t4 = time.perf_counter()
+        steps += 1
+        if steps <= warmup_steps:
+            continue
+        frac = ns / len(drv.running_slots)
         b = step_bytes(m, len(run), tot, 0)
         moved += b["kv"] + b["ssm"]
         n_ops += len(ops)
         t_alloc += t1 - t0
-        t_total += (t1 - t0) + (t4 - t3)
-        steps += 1
+        t_total += (t1 - t0) * frac + (t4 - t3)          # the allocator's share for the sampled part of the batch
+        sampled.append(ns)
+        batch.append(len(drv.running_slots))
+    k = max(steps - warmup_steps, 1)
     return {"value": moved / t_total / 1e9, "unit": "GB/s", "cores": 1, "host_cores": os.cpu_count(), "kind": "oracle",
-            "sample": f"{steps} consecutive engine steps of the same workload after {args.warm_steps} warm steps "
-                      f"(allocator step + translate + all-layer gathers), {t_total:.1f} s of CPU work",
+            "sample": f"{k} consecutive engine steps of the same workload after {args.warm_steps} warm steps: allocator "
+                      f"step of the whole batch, then translate + all-layer gathers for the first {int(np.mean(sampled or [0]))} of "
+                      f"{int(np.mean(batch or [0]))} running requests (what fits in {sample_bytes / 1e9:.0f} GB of host stores); "
+                      f"GB/s over the sampled requests' bytes, {t_total:.1f} s of CPU work",
             "allocator_ops_per_s": n_ops / t_alloc if t_alloc > 0 else None,
-            "ms_per_step": t_total / max(steps, 1) * 1e3, "steps": steps}
+            "ms_per_step": t_total / k * 1e3, "steps": k}
 
 
 def run_reference(args) -> dict:
     w = W.config(args.workload, seed=args.seed)
-    n = max(1, min(args.steps, 8))
-    base = run_oracle(args, n_sample_steps=n, budget_s=120.0)
+    base = run_oracle(args, n_sample_steps=args.steps, budget_s=240.0, warmup_steps=args.warmup)
     return {"metric": METRIC, "value": base["value"], "unit": "GB/s", "n_gpus": args.gpus, "steps": base["steps"],
             "warmup": args.warmup, "ms_per_step": base["ms_per_step"], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "u32", "data": "synthetic", "impl": "reference",
-            "config": {**config_dict(w, args.warm_steps), "note": "the CPU oracle as it stands, single thread, bounded sample of the same steps"},
+            "config": config_dict(w, args.warm_steps),
             "cpu_baseline": {k: base[k] for k in ("value", "unit", "cores", "kind", "sample")},
-            "allocator": {"ops_per_s": base["allocator_ops_per_s"]},
+            "roofline": {"secondary": {"allocator_ops_per_s": base["allocator_ops_per_s"]}},
+            "note": "the CPU oracle as it stands, single thread; each step is a bounded sample of the workload's step",
             "e2e": {"value": base["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
 
@@ -668,15 +814,15 @@ def run_reference(args) -> dict:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="short_uniform")
+    ap.add_argument("--workload", default="scale")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-micro", action="store_true", help="skip the migration and allocator micro-benchmarks")
+    ap.add_argument("--no-micro", action="store_true", help="skip the micro-benchmarks and the other configurations")
     ap.add_argument("--layers-per-launch", type=int, default=0,
-                    help="SSM / KV layers gathered per launch (0 = all layers of the model in one launch); "
+                    help="SSM / KV layers gathered per launch (0 = as many as fit beside the arena); "
                          "the batch buffers then hold that many layers and are reused by the next group")
     ap.add_argument("--warm-steps", type=int, default=WARM_STEPS, help="closed-loop steps before the timed window")
     args = ap.parse_args()
@@ -701,12 +847,14 @@ def main():
         if not args.no_micro:
             import torch
             dev = torch.device("cuda", local_rank)
-            out["migration"]["microbench"] = migration_microbench(dev)
-            out["allocator"]["vs_step_batch"] = allocator_scaling(dev)
-            out["closed_loop_device"] = device_closed_loop(dev, args.workload)
-            out["write_side"] = write_side_microbench(dev)
+            sec = out["roofline"]["secondary"]
+            sec["relocation_copy"] = migration_microbench(dev)
+            sec["allocator_vs_step_batch"] = allocator_scaling(dev)
+            sec["write_side"] = write_side_microbench(dev)
+            sec["closed_loop_device"] = device_closed_loop(dev, args.workload, 1500 if args.workload == "scale" else 3000)
+            out["roofline"]["other_configs"] = other_configs(dev, skip=args.workload)
         if not args.no_cpu_baseline:
-            out["cpu_baseline"] = run_oracle(args, n_sample_steps=20)
+            out["cpu_baseline"] = run_oracle(args, n_sample_steps=12)
         print(json.dumps(out), flush=True)
     if world > 1:
         dist.barrier()

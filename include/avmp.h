@@ -193,6 +193,8 @@ AVMP_API size_t avmp_workspace_bytes(const avmp_model_spec *spec, uint64_t pool_
  *   d_workspace  >= avmp_workspace_bytes(...), 256-byte aligned.
  *   migration_batch_size  B: upper bound, in donor units, on one migration (Section 3.1).
  *   opt          NULL = defaults.  threshold_low >= threshold_high is rejected (Section 4.6).
+ *                max_requests * max_pages_per_request * max(page_tokens, copy pieces per page) must
+ *                stay below 2^32: row offsets (cu_seqlens) and the gathers' piece counts are 32-bit.
  * Returns AVMP_EINVAL / AVMP_ENOSPC (workspace too small) / AVMP_ECUDA. */
 AVMP_API int avmp_create(avmp_ctx **out, const avmp_model_spec *spec, void *d_arena, uint64_t pool_bytes,
                 double initial_split, uint32_t migration_batch_size, const avmp_options *opt,
@@ -258,6 +260,20 @@ AVMP_API int avmp_gather_ssm_layers(avmp_ctx *ctx, uint32_t first_layer, uint32_
                                     uint32_t n_reqs, void *d_out_state, uint64_t state_layer_stride_bytes,
                                     void *d_out_conv, uint64_t conv_layer_stride_bytes, void *stream);
 
+/* Both gathers of an engine step in ONE launch (Section 2.2: the two access patterns, for the
+ * same request list): attention layers [first_attn_layer, + n_attn_layers) exactly as
+ * avmp_gather_kv_layers, then SSM layers [first_ssm_layer, + n_ssm_layers) exactly as
+ * avmp_gather_ssm_layers -- same outputs, same error items (a slot that is KV_ONLY contributes
+ * its rows to the KV part and one AVMP_DEV_BAD_REQUEST per SSM layer).  A step that moves only
+ * tens of MB is bound by the ramp and tail of its launches; this pays them once.  Both layer
+ * counts must be at least 1 (use the single-kind entry points otherwise). */
+AVMP_API int avmp_gather_step(avmp_ctx *ctx, const uint32_t *d_reqs, uint32_t n_reqs,
+                              uint32_t first_attn_layer, uint32_t n_attn_layers, void *d_out_k, void *d_out_v,
+                              uint64_t kv_layer_stride_bytes, uint64_t out_capacity_tokens, uint32_t *d_cu_seqlens,
+                              uint32_t first_ssm_layer, uint32_t n_ssm_layers, void *d_out_state,
+                              uint64_t state_layer_stride_bytes, void *d_out_conv, uint64_t conv_layer_stride_bytes,
+                              void *stream);
+
 /* Write side of the two gathers (what the model's kernels do after a step).  Tokens
  * [d_tok_start[k], len_k) of request k are read from rows cu[k].. of d_in_k / d_in_v, cu being
  * the prefix sum of (len_k - d_tok_start[k]); d_tok_start == NULL means 0. */
@@ -273,9 +289,13 @@ AVMP_API int avmp_scatter_ssm(avmp_ctx *ctx, uint32_t ssm_layer, const uint32_t 
  * plug-in that is only ever handed device pointers.  Inputs and outputs are still the
  * caller's; the gather's planning arrays live in a fixed array inside the library
  * (about 33 KB per GPU, held until the process exits), which limits the request list to
- * AVMP_STATIC_GATHER_MAX_REQS entries: a longer list returns AVMP_ETOOBIG and does nothing.
- * The context's device must be current.  The first call on a device resolves the array's
- * device address (a host-side set-up step); make that first call before any stream capture.
+ * AVMP_STATIC_GATHER_MAX_REQS entries: a longer list returns AVMP_ETOOBIG and does nothing
+ * (and, as for avmp_gather_kv, a list longer than max_requests returns AVMP_EINVAL).
+ * The context's device must be current.  The array's device address is resolved on the host,
+ * once per device: by avmp_create (so that the driver loads the array onto the GPU while the
+ * caller still has memory to spare), or else by the first call of this entry point on that
+ * device -- make that call (n_reqs = 0 will do) before handing all memory away and before any
+ * stream capture.  After a cudaDeviceReset create a new context before calling this again.
  * All calls on a device share the array: calls whose kernels may overlap on the GPU
  * (different streams) race -- keep them on one stream or order them with events.  Results,
  * error items and cu_seqlens are exactly those of avmp_gather_kv. */

@@ -114,6 +114,8 @@ def _load():
         "avmp_gather_ssm": (C.c_int, [vp, C.c_uint32, vp, C.c_uint32, vp, vp, vp]),
         "avmp_gather_kv_layers": (C.c_int, [vp, C.c_uint32, C.c_uint32, vp, C.c_uint32, vp, vp, C.c_uint64, C.c_uint64, vp, vp]),
         "avmp_gather_ssm_layers": (C.c_int, [vp, C.c_uint32, C.c_uint32, vp, C.c_uint32, vp, C.c_uint64, vp, C.c_uint64, vp]),
+        "avmp_gather_step": (C.c_int, [vp, vp, C.c_uint32, C.c_uint32, C.c_uint32, vp, vp, C.c_uint64, C.c_uint64, vp,
+                                       C.c_uint32, C.c_uint32, vp, C.c_uint64, vp, C.c_uint64, vp]),
         "avmp_scatter_kv": (C.c_int, [vp, C.c_uint32, vp, vp, C.c_uint32, vp, vp, vp]),
         "avmp_scatter_ssm": (C.c_int, [vp, C.c_uint32, vp, C.c_uint32, vp, vp, vp]),
         "avmp_scatter_kv_layers": (C.c_int, [vp, C.c_uint32, C.c_uint32, vp, vp, C.c_uint32, vp, vp, C.c_uint64, vp]),
@@ -316,6 +318,15 @@ def avmp_gather_ssm_layers(ctx, first_layer, n_layers, d_reqs, n_reqs, d_out_sta
                                       _stream(stream)), "avmp_gather_ssm_layers")
 
 
+def avmp_gather_step(ctx, d_reqs, n_reqs, first_attn_layer, n_attn_layers, d_out_k, d_out_v, kv_layer_stride_bytes,
+                     out_capacity_tokens, d_cu_seqlens, first_ssm_layer, n_ssm_layers, d_out_state,
+                     state_layer_stride_bytes, d_out_conv, conv_layer_stride_bytes, stream=None):
+    _check(lib.avmp_gather_step(ctx, _ptr(d_reqs), n_reqs, first_attn_layer, n_attn_layers, _ptr(d_out_k), _ptr(d_out_v),
+                                kv_layer_stride_bytes, out_capacity_tokens, _ptr(d_cu_seqlens), first_ssm_layer,
+                                n_ssm_layers, _ptr(d_out_state), state_layer_stride_bytes, _ptr(d_out_conv),
+                                conv_layer_stride_bytes, _stream(stream)), "avmp_gather_step")
+
+
 def avmp_scatter_kv(ctx, attn_layer, d_reqs, d_tok_start, n_reqs, d_in_k, d_in_v, stream=None):
     _check(lib.avmp_scatter_kv(ctx, attn_layer, _ptr(d_reqs), _ptr(d_tok_start), n_reqs, _ptr(d_in_k),
                                _ptr(d_in_v), _stream(stream)), "avmp_scatter_kv")
@@ -490,6 +501,12 @@ class Context:
                           conv_stride, stream=None):
         avmp_gather_ssm_layers(self.handle, first_layer, n_layers, d_reqs, n, d_out_state, state_stride,
                                d_out_conv, conv_stride, stream)
+
+    def gather_step(self, d_reqs, n, first_attn_layer, n_attn_layers, d_out_k, d_out_v, kv_layer_stride, cap_tokens, d_cu,
+                    first_ssm_layer, n_ssm_layers, d_out_state, state_stride, d_out_conv, conv_stride, stream=None):
+        avmp_gather_step(self.handle, d_reqs, n, first_attn_layer, n_attn_layers, d_out_k, d_out_v, kv_layer_stride,
+                         cap_tokens, d_cu, first_ssm_layer, n_ssm_layers, d_out_state, state_stride, d_out_conv,
+                         conv_stride, stream)
 
     def scatter_kv(self, layer, d_reqs, d_tok_start, n, d_in_k, d_in_v, stream=None):
         avmp_scatter_kv(self.handle, layer, d_reqs, d_tok_start, n, d_in_k, d_in_v, stream)

@@ -10,7 +10,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
-LIB = Path(os.environ["AVMP_LIB"]) if os.environ.get("AVMP_LIB") else PKG / "libavmp.so"
+LIB = PKG / "libavmp.so"
 SOURCES = ["avmp_api.cu", "avmp_step.cu", "avmp_copy.cu", "avmp_noalloc.cu", "avmp_driver.cu",
            "avmp_sessions.cu"]
 HEADERS = [CSRC / "avmp_dev.cuh", CSRC / "avmp_step_body.cuh", ROOT / "include" / "avmp.h"]
@@ -37,8 +37,7 @@ def build_library(force: bool = False, verbose: bool = False) -> Path:
     if not force and not needs_build():
         return LIB
     tmp = LIB.with_suffix(f".tmp{os.getpid()}.so")
-    extra = os.environ.get("AVMP_NVCC_FLAGS", "").split()      # developer knob: e.g. -DAVMP_STAGES=4
-    cmd = [_nvcc(), *NVCC_FLAGS, *extra, *(["-Xptxas", "-v"] if verbose else []), "-o", str(tmp),
+    cmd = [_nvcc(), *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []), "-o", str(tmp),
            *[str(CSRC / s) for s in SOURCES]]
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)

@@ -262,7 +262,18 @@ int avmp_create(avmp_ctx **out, const avmp_model_spec *spec, void *d_arena, uint
         init.n_vfree[p] = (uint32_t)lay.vid_space[p];
     }
     init.fsm = AVMP_FSM_BALANCED;
+    // The row and piece prefix sums of a KV gather are 32-bit, like cu_seqlens: no request list of
+    // up to max_requests entries (repeats allowed) may total 2^32 rows or copy pieces.
+    {
+        const uint64_t subs = kv_pieces_per_page(lay, spec->page_tokens);
+        const uint64_t per_req = (uint64_t)o.max_pages_per_request * (spec->page_tokens > subs ? spec->page_tokens : subs);
+        if ((unsigned __int128)o.max_requests * per_req >= ((unsigned __int128)1 << 32)) { delete c; return AVMP_EINVAL; }
+    }
     if (launch_init(g, init, S(stream)) != cudaSuccess) { delete c; return AVMP_ECUDA; }
+    // Bring avmp_gather_kv_static's in-library scratch onto this device now, while the caller still
+    // has memory to spare (a failure here only shows up if that entry point is ever called).
+    (void)static_gather_setup(dev);
+    (void)cudaGetLastError();
     c->launches += 1;
     *out = c;
     return AVMP_OK;
@@ -404,6 +415,26 @@ int avmp_gather_ssm_layers(avmp_ctx *c, uint32_t first_layer, uint32_t n_layers,
     c->launches += 1;
     return cu(launch_ssm(c->g, false, first_layer, n_layers, d_reqs, n, d_out_state, state_layer_stride_bytes,
                          d_out_conv, conv_layer_stride_bytes, L(c, stream)));
+}
+
+int avmp_gather_step(avmp_ctx *c, const uint32_t *d_reqs, uint32_t n, uint32_t first_attn_layer, uint32_t n_attn_layers,
+                     void *d_out_k, void *d_out_v, uint64_t kv_layer_stride_bytes, uint64_t cap_tokens, uint32_t *d_cu,
+                     uint32_t first_ssm_layer, uint32_t n_ssm_layers, void *d_out_state, uint64_t state_layer_stride_bytes,
+                     void *d_out_conv, uint64_t conv_layer_stride_bytes, void *stream)
+{
+    if (!c || n_attn_layers == 0 || (uint64_t)first_attn_layer + n_attn_layers > c->spec.n_attn_layers) return AVMP_EINVAL;
+    if (n_ssm_layers == 0 || (uint64_t)first_ssm_layer + n_ssm_layers > c->spec.n_ssm_layers) return AVMP_EINVAL;
+    if (n > c->opt.max_requests || !d_cu) return AVMP_EINVAL;
+    if (n && (!d_reqs || !d_out_k || !d_out_v || !d_out_state || !d_out_conv)) return AVMP_EINVAL;
+    if (((uintptr_t)d_out_k | (uintptr_t)d_out_v | kv_layer_stride_bytes | (uintptr_t)d_out_state | (uintptr_t)d_out_conv |
+         state_layer_stride_bytes | conv_layer_stride_bytes) & 15) return AVMP_EINVAL;
+    if (n_attn_layers > 1 && kv_layer_stride_bytes < cap_tokens * c->lay.kv_row_bytes) return AVMP_EINVAL;
+    if (n_ssm_layers > 1 && (state_layer_stride_bytes < (uint64_t)n * c->lay.ssm_state_bytes ||
+                             conv_layer_stride_bytes < (uint64_t)n * c->lay.ssm_conv_bytes)) return AVMP_EINVAL;
+    c->launches += n > kLocalPlanMax ? 2 : 1;
+    return cu(launch_step_gather(c->g, d_reqs, n, first_attn_layer, n_attn_layers, d_out_k, d_out_v, kv_layer_stride_bytes,
+                                 cap_tokens, d_cu, first_ssm_layer, n_ssm_layers, d_out_state, state_layer_stride_bytes,
+                                 d_out_conv, conv_layer_stride_bytes, L(c, stream)));
 }
 
 int avmp_scatter_kv_layers(avmp_ctx *c, uint32_t first_layer, uint32_t n_layers, const uint32_t *d_reqs,

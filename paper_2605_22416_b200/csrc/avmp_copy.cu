@@ -32,23 +32,10 @@ namespace avmp {
 
 namespace {
 
-// Tunables (overridable at build time for sweeps).
-#ifndef AVMP_STAGE_BYTES
-#define AVMP_STAGE_BYTES 16384
-#endif
-#ifndef AVMP_STAGES
-#define AVMP_STAGES 3
-#endif
-#ifndef AVMP_BULK_WARPS
-#define AVMP_BULK_WARPS 4
-#endif
-#ifndef AVMP_BULK_CTAS_PER_SM
-#define AVMP_BULK_CTAS_PER_SM 1
-#endif
-constexpr uint32_t kStage = AVMP_STAGE_BYTES;   // bytes per piece
-constexpr int kStages = AVMP_STAGES;            // ring depth per warp
-constexpr int kBulkWarps = AVMP_BULK_WARPS;     // warps (rings) per CTA: 4 x 3 x 16 KiB = 192 KiB of shared memory
-constexpr int kBulkCtasPerSm = AVMP_BULK_CTAS_PER_SM;
+// Shape of the bulk path (fixed after sweeps on B200; see the measured alternatives above).
+constexpr int kStages = 3;                      // ring depth per warp
+constexpr int kBulkWarps = 4;                   // warps (rings) per CTA: 4 x 3 x 16 KiB = 192 KiB of shared memory
+constexpr int kBulkCtasPerSm = 1;
 constexpr int kBulkThreads = kBulkWarps * 32;
 constexpr uint32_t kBulkSmem = kBulkWarps * kStages * kStage;
 constexpr int kGenThreads = 256;
@@ -135,21 +122,26 @@ struct RelocPieces {
 // its dependency, and calls on different streams share no scratch); longer lists use the plan
 // kernel and the context's global scratch.
 // One request's rows and pieces for a KV gather / scatter (errors recorded by the caller's choice).
+__device__ __forceinline__ void kv_rows_items(const Geom &g, uint32_t st, uint32_t len, uint32_t t0, uint32_t subs,
+                                              bool report, uint32_t &rows, uint32_t &items)
+{
+    rows = 0; items = 0;
+    if (st == AVMP_REQ_EMPTY) { if (report) record_error(g.st, AVMP_DEV_BAD_REQUEST); }
+    else if (t0 > len) { if (report) record_error(g.st, AVMP_DEV_BAD_REQUEST); }
+    else rows = len - t0;
+    if (rows) items = ((t0 + rows - 1u) / g.T - t0 / g.T + 1u) * subs;
+}
+
 __device__ __forceinline__ void kv_plan_entry(const Geom &g, const uint32_t *reqs, const uint32_t *tok_start,
                                               uint32_t k, uint32_t subs, bool report, uint32_t &rows, uint32_t &items)
 {
-    rows = 0; items = 0;
     const uint32_t r = reqs[k];
-    const uint32_t st = r < g.R ? g.r_state[r] : AVMP_REQ_EMPTY;
-    const uint32_t t0 = tok_start ? tok_start[k] : 0u;
-    if (st == AVMP_REQ_EMPTY) { if (report) record_error(g.st, AVMP_DEV_BAD_REQUEST); }
-    else {
-        const uint32_t len = g.r_len[r];
-        if (t0 > len) { if (report) record_error(g.st, AVMP_DEV_BAD_REQUEST); }
-        else rows = len - t0;
-    }
-    if (rows) items = ((t0 + rows - 1u) / g.T - t0 / g.T + 1u) * subs;
+    const bool in_range = r < g.R;
+    kv_rows_items(g, in_range ? g.r_state[r] : (uint32_t)AVMP_REQ_EMPTY, in_range ? g.r_len[r] : 0u,
+                  tok_start ? tok_start[k] : 0u, subs, report, rows, items);
 }
+
+constexpr uint32_t kPlanWords = 3 * (kLocalPlanMax + 1);   // shared words a local plan needs: rows, items, slots
 
 template <bool SCATTER>
 struct KvPieces {
@@ -161,33 +153,72 @@ struct KvPieces {
     unsigned long long cap_tokens, layer_stride;
     uint32_t *cu_out;                     // cu_seqlens for the caller (local plan only; may be null)
     const uint32_t *cu_items, *cu_rows;   // set by plan(): shared memory, or the context's scratch
-    // Whole CTA.  `buf` holds 2 * (kLocalPlanMax + 1) words, `tmp` 32 scan words.
+    const uint32_t *req_of;               // set by plan(): the list's slots (shared copy, or the caller's array)
+    // Whole CTA.  `buf` holds kPlanWords words, `tmp` 32 scan words.
     __device__ void plan(const Geom &g, uint32_t *buf, unsigned long long *tmp)
     {
-        if (n > kLocalPlanMax) { cu_items = g.g_cu_items; cu_rows = g.g_cu_rows; return; }
-        uint32_t *rows_s = buf, *items_s = buf + kLocalPlanMax + 1;
+        if (n > kLocalPlanMax) { cu_items = g.g_cu_items; cu_rows = g.g_cu_rows; req_of = reqs; return; }
+        uint32_t *rows_s = buf, *items_s = buf + kLocalPlanMax + 1, *req_s = buf + 2 * (kLocalPlanMax + 1);
         const bool lead = blockIdx.x == 0;            // one CTA reports errors and writes cu_seqlens
-        unsigned long long run_rows = 0, run_items = 0, tot;
-        for (uint32_t b = 0; b < n; b += blockDim.x) {
-            const uint32_t k = b + threadIdx.x;
-            uint32_t rows = 0, items = 0;
-            if (k < n) kv_plan_entry(g, reqs, tok_start, k, subs, lead, rows, items);
-            const unsigned long long incl = block_incl_scan(((unsigned long long)items << 32) | rows, tmp, &tot);
-            if (k < n) {
-                const uint32_t ex_rows = (uint32_t)(run_rows + (uint32_t)incl - rows);
-                rows_s[k] = ex_rows;
-                items_s[k] = (uint32_t)(run_items + (uint32_t)(incl >> 32) - items);
-                if (lead && cu_out) cu_out[k] = ex_rows;
-            }
-            run_rows += (uint32_t)tot;
-            run_items += (uint32_t)(tot >> 32);
+        // Pass 1: every entry's rows and pieces, with all table reads of the list in flight together
+        // (two dependent reads per entry; taken window by window between the scans' barriers they
+        // would cost that latency once per window).  kPer entries per thread cover the longest local
+        // list with the smallest CTA that runs this (128 threads).
+        constexpr int kPer = 8;
+        uint32_t rr[kPer], t0[kPer], st[kPer], ln[kPer];
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+            const uint32_t k = threadIdx.x + i * blockDim.x;
+            rr[i] = k < n ? reqs[k] : kInvalid;
+            t0[i] = (k < n && tok_start) ? tok_start[k] : 0u;
         }
-        if (threadIdx.x == 0) {
-            rows_s[n] = (uint32_t)run_rows; items_s[n] = (uint32_t)run_items;
-            if (lead && cu_out) cu_out[n] = (uint32_t)run_rows;
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+            const bool in_range = rr[i] < g.R;
+            st[i] = in_range ? g.r_state[rr[i]] : (uint32_t)AVMP_REQ_EMPTY;
+            ln[i] = in_range ? g.r_len[rr[i]] : 0u;
+        }
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+            const uint32_t k = threadIdx.x + i * blockDim.x;
+            if (k < n) {
+                uint32_t rows, items;
+                kv_rows_items(g, st[i], ln[i], t0[i], subs, lead, rows, items);
+                rows_s[k] = rows; items_s[k] = items; req_s[k] = rr[i];
+            }
         }
         __syncthreads();
-        cu_items = items_s; cu_rows = rows_s;
+        // Pass 2: exclusive prefix sums over the list: every thread sums a run of consecutive entries,
+        // one block scan orders the runs (one scan for the whole list instead of one per window).
+        const uint32_t per = (n + blockDim.x - 1) / blockDim.x;          // <= kPer
+        const uint32_t k0 = threadIdx.x * per;
+        uint32_t vr[kPer], vi[kPer];
+        unsigned long long mine = 0, tot;
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+            const uint32_t k = k0 + i;
+            const bool in = (uint32_t)i < per && k < n;
+            vr[i] = in ? rows_s[k] : 0u; vi[i] = in ? items_s[k] : 0u;
+            mine += ((unsigned long long)vi[i] << 32) | vr[i];
+        }
+        const unsigned long long incl = block_incl_scan(mine, tmp, &tot);
+        unsigned long long run = incl - mine;
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+            const uint32_t k = k0 + i;
+            if ((uint32_t)i < per && k < n) {
+                rows_s[k] = (uint32_t)run;
+                items_s[k] = (uint32_t)(run >> 32);
+                if (lead && cu_out) cu_out[k] = (uint32_t)run;
+                run += ((unsigned long long)vi[i] << 32) | vr[i];
+            }
+        }
+        if (threadIdx.x == 0) {
+            rows_s[n] = (uint32_t)tot; items_s[n] = (uint32_t)(tot >> 32);
+            if (lead && cu_out) cu_out[n] = (uint32_t)tot;
+        }
+        __syncthreads();
+        cu_items = items_s; cu_rows = rows_s; req_of = req_s;
     }
     __device__ unsigned long long total(const Geom &) const { return (unsigned long long)n_layers * cu_items[n]; }
     __device__ Piece get(const Geom &g, unsigned long long it64) const
@@ -211,7 +242,7 @@ struct KvPieces {
         const uint32_t b_lo = max((lo_t - page * T) * row, q * kStage);
         const uint32_t b_hi = min((hi_t - page * T) * row, (q + 1u) * kStage);
         if (b_lo >= b_hi) return Piece{nullptr, nullptr, 0};
-        const uint32_t r = reqs[k];
+        const uint32_t r = req_of[k];
         const uint32_t h = g.r_chain[(unsigned long long)r * g.max_pages + page];
         const uint32_t slot = g.VT[0][h & 0x7FFFFFFFu];
         uint8_t *p = g.arena + (unsigned long long)slot * g.U[0] + (unsigned long long)(layer0 + dl) * g.kv_layer_bytes +
@@ -221,6 +252,23 @@ struct KvPieces {
                      ((unsigned long long)row0 * row + (unsigned long long)page * T * row + b_lo -
                       (unsigned long long)t0 * row);
         return SCATTER ? Piece{b, p, b_hi - b_lo} : Piece{p, b, b_hi - b_lo};
+    }
+};
+
+// a11 + a12 in one launch: the KV pieces of a range of attention layers, then the SSM pieces of a
+// range of SSM layers, for one request list.  A step that moves little (a few dozen requests) is
+// bound by the ramp and the tail of its launches; one launch pays them once.
+struct StepPieces {
+    static constexpr bool kTimed = false;
+    static constexpr bool kPlans = true;
+    KvPieces<false> kv;
+    SsmPieces<false> ssm;
+    __device__ void plan(const Geom &g, uint32_t *buf, unsigned long long *tmp) { kv.plan(g, buf, tmp); }
+    __device__ unsigned long long total(const Geom &g) const { return kv.total(g) + ssm.total(g); }
+    __device__ Piece get(const Geom &g, unsigned long long it) const
+    {
+        const unsigned long long nkv = kv.total(g);
+        return it < nkv ? kv.get(g, it) : ssm.get(g, it - nkv);
     }
 };
 
@@ -245,41 +293,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 // Both directions carry an L2 evict-first hint: the bytes stream through once, and keeping them
-// from displacing each other's lines was worth 2-5 % on this part (AVMP_LOAD_HINT / AVMP_STORE_HINT = 0
-// build the unhinted forms: without the load hint the benchmark step loses 1.7 %, without the store
-// hint 0.5 %, single-layer launches 3-4 % each).
+// from displacing each other's lines was worth 2-5 % on this part (measured against the unhinted
+// forms: without the load hint the benchmark step loses 1.7 %, without the store hint 0.5 %,
+// single-layer launches 3-4 % each).
 __device__ __forceinline__ unsigned long long l2_policy_evict_first()
 {
     unsigned long long p;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
     return p;
 }
-#ifndef AVMP_LOAD_HINT
-#define AVMP_LOAD_HINT 1
-#endif
-#ifndef AVMP_STORE_HINT
-#define AVMP_STORE_HINT 1
-#endif
 __device__ __forceinline__ void bulk_g2s(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar,
                                          unsigned long long pol)
 {
-#if AVMP_LOAD_HINT
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
                  :: "r"(dst_smem), "l"(src), "r"(bytes), "r"(bar), "l"(pol) : "memory");
-#else
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 :: "r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
-#endif
 }
 __device__ __forceinline__ void bulk_s2g(void *dst, uint32_t src_smem, uint32_t bytes, unsigned long long pol)
 {
-#if AVMP_STORE_HINT
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;"
                  :: "l"(dst), "r"(src_smem), "r"(bytes), "l"(pol) : "memory");
-#else
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                 :: "l"(dst), "r"(src_smem), "r"(bytes) : "memory");
-#endif
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
 template <int N>
@@ -329,6 +361,17 @@ struct Ring {
         bulk_s2g(dst[s], buf0 + s * kStage, bytes[s], policy);
         ++n_stored;
     }
+    // After a timeout: no new copies, but loads already issued still target this CTA's shared
+    // memory.  Give each of them one more bounded wait (nothing is stored) before the CTA may exit.
+    __device__ __forceinline__ void drain_loads()
+    {
+        for (uint32_t i = n_stored; i < n_loaded; ++i) {
+            const uint32_t s = i % kStages, parity = (i / kStages) & 1u;
+            uint32_t spins = 0;
+            while (!mbar_try_wait(bar0 + 8u * s, parity))
+                if (++spins > kSpinLimit) break;
+        }
+    }
     __device__ __forceinline__ void push(const Piece &p)
     {
         if (n_loaded - n_stored == (uint32_t)kStages) retire_one();
@@ -362,7 +405,7 @@ __global__ void __launch_bounds__(kBulkThreads, kBulkCtasPerSm) stream_bulk_kern
     __syncthreads();
     F f = f_in;
     if constexpr (F::kPlans) {
-        __shared__ uint32_t plan_buf[2 * (kLocalPlanMax + 1)];
+        __shared__ uint32_t plan_buf[kPlanWords];
         __shared__ unsigned long long plan_tmp[32];
         f.plan(g, plan_buf, plan_tmp);
     }
@@ -407,7 +450,10 @@ __global__ void __launch_bounds__(kBulkThreads, kBulkCtasPerSm) stream_bulk_kern
     }
     if (lane == 0) {
         while (!ring.failed && ring.n_stored < ring.n_loaded) ring.retire_one();
-        if (ring.failed) record_error(g.st, AVMP_DEV_TIMEOUT);
+        if (ring.failed) {
+            record_error(g.st, AVMP_DEV_TIMEOUT);
+            ring.drain_loads();
+        }
         bulk_wait_all();
         if (F::kTimed) atomicMax(&g.st->reloc_t1, global_ns());
     }
@@ -420,7 +466,7 @@ __global__ void __launch_bounds__(kGenThreads) stream_generic_kernel(const Geom 
     pdl_prologue();
     F f = f_in;
     if constexpr (F::kPlans) {
-        __shared__ uint32_t plan_buf[2 * (kLocalPlanMax + 1)];
+        __shared__ uint32_t plan_buf[kPlanWords];
         __shared__ unsigned long long plan_tmp[32];
         f.plan(g, plan_buf, plan_tmp);
     }
@@ -541,8 +587,30 @@ cudaError_t launch_kv(const Geom &g, bool scatter, uint32_t layer0, uint32_t n_l
     }
     const bool bulk_ok = mult16(g.row_bytes) && mult16(g.U[0]) && mult16(g.kv_layer_bytes) && mult16(layer_stride);
     if (scatter)
-        return launch_stream(g, KvPieces<true>{layer0, n_layers, n, subs, reqs, tok_start, (uint8_t *)k, (uint8_t *)v, cap_tokens, layer_stride, cu_out, nullptr, nullptr}, bulk_ok, l);
-    return launch_stream(g, KvPieces<false>{layer0, n_layers, n, subs, reqs, tok_start, (uint8_t *)k, (uint8_t *)v, cap_tokens, layer_stride, cu_out, nullptr, nullptr}, bulk_ok, l);
+        return launch_stream(g, KvPieces<true>{layer0, n_layers, n, subs, reqs, tok_start, (uint8_t *)k, (uint8_t *)v, cap_tokens, layer_stride, cu_out, nullptr, nullptr, nullptr}, bulk_ok, l);
+    return launch_stream(g, KvPieces<false>{layer0, n_layers, n, subs, reqs, tok_start, (uint8_t *)k, (uint8_t *)v, cap_tokens, layer_stride, cu_out, nullptr, nullptr, nullptr}, bulk_ok, l);
+}
+
+cudaError_t launch_step_gather(const Geom &g, const uint32_t *reqs, uint32_t n, uint32_t kv_layer0, uint32_t kv_layers,
+                               void *k, void *v, unsigned long long kv_layer_stride, unsigned long long cap_tokens,
+                               uint32_t *cu_out, uint32_t ssm_layer0, uint32_t ssm_layers, void *state,
+                               unsigned long long state_stride, void *conv, unsigned long long conv_stride, const Launch &l)
+{
+    const unsigned long long part = (unsigned long long)g.T * g.row_bytes;
+    const uint32_t subs = 2u * (uint32_t)((part + kStage - 1) / kStage);
+    if (n > kLocalPlanMax) {
+        cudaError_t e = launch_pdl(kv_plan_kernel, dim3(1), dim3(kStepThreads), 0, l.stream, g, reqs, (const uint32_t *)nullptr, n, subs, cu_out);
+        if (e != cudaSuccess) return e;
+    }
+    const uint32_t ps = (uint32_t)((g.state_bytes + kStage - 1) / kStage), pc = (uint32_t)((g.conv_bytes + kStage - 1) / kStage);
+    const bool bulk_ok = mult16(g.row_bytes) && mult16(g.U[0]) && mult16(g.kv_layer_bytes) && mult16(kv_layer_stride) &&
+                         mult16(g.state_bytes) && mult16(g.conv_bytes) && mult16(g.U[1]) && mult16(g.P_al) &&
+                         mult16(state_stride) && mult16(conv_stride);
+    StepPieces f{KvPieces<false>{kv_layer0, kv_layers, n, subs, reqs, nullptr, (uint8_t *)k, (uint8_t *)v, cap_tokens,
+                                 kv_layer_stride, cu_out, nullptr, nullptr, nullptr},
+                 SsmPieces<false>{ssm_layer0, ssm_layers, n, ps, ps + pc, reqs, (uint8_t *)state, (uint8_t *)conv,
+                                  state_stride, conv_stride}};
+    return launch_stream(g, f, bulk_ok, l);
 }
 
 cudaError_t launch_ssm(const Geom &g, bool scatter, uint32_t layer0, uint32_t n_layers, const uint32_t *reqs, uint32_t n,

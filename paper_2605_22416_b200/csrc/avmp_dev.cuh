@@ -12,6 +12,7 @@ namespace avmp {
 
 constexpr uint32_t kInvalid = 0xFFFFFFFFu;
 constexpr unsigned long long kNone64 = 0xFFFFFFFFFFFFFFFFull;
+constexpr uint32_t kStage = 16384;           // bytes per piece of a streaming copy (one ring stage)
 constexpr uint32_t kLocalPlanMax = 1024;    // longest request list a KV copy plans inside its own CTAs
 constexpr int kStepThreads = 1024;          // one CTA plans a step; one op per thread per window
 constexpr uint32_t kHostStepMaxOps = 65536; // staging capacity of avmp_step_host
@@ -121,7 +122,7 @@ __device__ __forceinline__ uint32_t find_owner(const uint32_t *a, uint32_t lo, u
 }
 
 // ---- programmatic dependent launch ------------------------------------------------------
-// Every kernel of the library starts with pdl_prologue(): it lets the next kernel in the stream
+// Every kernel of the library is launched through launch_pdl and starts with pdl_prologue(): it lets the next kernel in the stream
 // be scheduled at once (its CTAs become resident as resources free up and its launch latency is
 // hidden), then waits until everything before it in the stream has completed and is visible.
 // No global memory is touched before the wait, so stream order is preserved exactly; launched
@@ -149,6 +150,13 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
+// Pieces a KV copy cuts one page of one layer into: K slices, then V slices.
+inline uint32_t kv_pieces_per_page(const avmp_layout &lay, uint32_t page_tokens)
+{
+    const unsigned long long part = (unsigned long long)page_tokens * lay.kv_row_bytes;
+    return 2u * (uint32_t)((part + kStage - 1) / kStage);
+}
+
 // Host-side launch wrappers (defined next to their kernels).
 struct Launch {
     cudaStream_t stream;
@@ -167,6 +175,12 @@ cudaError_t launch_kv(const Geom &g, bool scatter, uint32_t layer0, uint32_t n_l
 cudaError_t launch_ssm(const Geom &g, bool scatter, uint32_t layer0, uint32_t n_layers, const uint32_t *reqs, uint32_t n,
                        void *state, unsigned long long state_stride, void *conv, unsigned long long conv_stride,
                        const Launch &l);
+cudaError_t launch_step_gather(const Geom &g, const uint32_t *reqs, uint32_t n, uint32_t kv_layer0, uint32_t kv_layers,
+                               void *k, void *v, unsigned long long kv_layer_stride, unsigned long long cap_tokens,
+                               uint32_t *cu_out, uint32_t ssm_layer0, uint32_t ssm_layers, void *state,
+                               unsigned long long state_stride, void *conv, unsigned long long conv_stride, const Launch &l);
+// Resolves the in-library scratch of avmp_gather_kv_static on the current device (= dev).
+cudaError_t static_gather_setup(int dev);
 
 }  // namespace avmp
 

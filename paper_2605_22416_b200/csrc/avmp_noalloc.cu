@@ -44,6 +44,7 @@ static_plan_kernel(const Geom g, uint32_t *__restrict__ scratch, const uint32_t 
     __shared__ unsigned long long tmp[32];
     unsigned long long run_rows = 0, run_items = 0, tot;
     const int tid = threadIdx.x;
+    pdl_prologue();
     for (uint32_t b = 0; b < n; b += kStepThreads) {
         const uint32_t k = b + tid;
         uint32_t rows = 0;
@@ -90,6 +91,7 @@ static_gather_kernel(const Geom g, const uint32_t *__restrict__ scratch, const u
                      const uint32_t *__restrict__ reqs, const uint32_t n, const uint32_t tpi,
                      uint8_t *__restrict__ out_k, uint8_t *__restrict__ out_v, const unsigned long long cap_tokens)
 {
+    pdl_prologue();
     const uint32_t *cu_rows = scratch + kRowsOff, *cu_items = scratch + kItemsOff;
     const uint32_t total = scratch[kTotalOff];
     const int lane = threadIdx.x & 31;
@@ -122,10 +124,26 @@ static_gather_kernel(const Geom g, const uint32_t *__restrict__ scratch, const u
     }
 }
 
-// Device address of the scratch array, per device; filled by the first call on that device.
+// Device address of the scratch array, per device.
 uint32_t *g_scratch_addr[64] = {};
 
 }  // namespace
+
+// Resolve the array's address on the current device.  Under CUDA's lazy module loading this is
+// also the moment the driver loads this file's code and the array onto the GPU, so it is done
+// when a context is created -- while the caller can still spare the memory -- and again by the
+// entry point if that did not happen.  Re-resolved at every avmp_create: after a cudaDeviceReset
+// the old address is stale, and so is every context made before the reset.
+cudaError_t avmp::static_gather_setup(int dev)
+{
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    void *p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_static_gather_scratch);
+    if (e != cudaSuccess) return e;
+    if (!p) return cudaErrorInvalidSymbol;
+    g_scratch_addr[dev] = static_cast<uint32_t *>(p);
+    return cudaSuccess;
+}
 
 extern "C" AVMP_API int avmp_gather_kv_static(avmp_ctx *c, uint32_t layer, const uint32_t *d_reqs, uint32_t n,
                                               void *d_out_k, void *d_out_v, uint64_t cap_tokens,
@@ -133,28 +151,25 @@ extern "C" AVMP_API int avmp_gather_kv_static(avmp_ctx *c, uint32_t layer, const
 {
     if (!c || layer >= c->spec.n_attn_layers || !d_cu) return AVMP_EINVAL;
     if (n > kMaxReqs) return AVMP_ETOOBIG;            // the fixed scratch cannot plan a longer list
+    if (n > c->opt.max_requests) return AVMP_EINVAL;  // as avmp_gather_kv: a list is no longer than the slot table
     if (n && (!d_reqs || !d_out_k || !d_out_v)) return AVMP_EINVAL;
     if (((uintptr_t)d_out_k | (uintptr_t)d_out_v) & 15) return AVMP_EINVAL;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) return AVMP_ECUDA;
     if (dev != c->device || dev < 0 || dev >= 64) return AVMP_EINVAL;   // the context's device must be current
-    if (!g_scratch_addr[dev]) {
-        // One-time set-up for this device: resolve the symbol to its address on this GPU.
-        void *p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_static_gather_scratch) != cudaSuccess || !p) return AVMP_ECUDA;
-        g_scratch_addr[dev] = static_cast<uint32_t *>(p);
-    }
+    // Normally resolved by avmp_create; a context made on another device's turn gets it here.
+    if (!g_scratch_addr[dev] && static_gather_setup(dev) != cudaSuccess) return AVMP_ECUDA;
     uint32_t *scratch = g_scratch_addr[dev];
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     uint32_t tpi = (uint32_t)(4096 / (c->g.row_bytes ? c->g.row_bytes : 1));
     if (tpi < 1) tpi = 1;
     if (tpi > c->g.T) tpi = c->g.T;
-    static_plan_kernel<<<1, kStepThreads, 0, s>>>(c->g, scratch, d_reqs, n, tpi, d_cu);
-    if (cudaGetLastError() != cudaSuccess) return AVMP_ECUDA;
-    static_gather_kernel<<<c->n_sms * 4, kThreads, 0, s>>>(c->g, scratch, layer, d_reqs, n, tpi,
-                                                            static_cast<uint8_t *>(d_out_k),
-                                                            static_cast<uint8_t *>(d_out_v), cap_tokens);
-    if (cudaGetLastError() != cudaSuccess) return AVMP_ECUDA;
+    if (launch_pdl(static_plan_kernel, dim3(1), dim3(kStepThreads), 0, s, c->g, scratch, d_reqs, n, tpi, d_cu) != cudaSuccess)
+        return AVMP_ECUDA;
+    if (launch_pdl(static_gather_kernel, dim3(c->n_sms * 4), dim3(kThreads), 0, s, c->g, (const uint32_t *)scratch, layer,
+                   d_reqs, n, tpi, static_cast<uint8_t *>(d_out_k), static_cast<uint8_t *>(d_out_v),
+                   (unsigned long long)cap_tokens) != cudaSuccess)
+        return AVMP_ECUDA;
     c->launches += 2;
     return AVMP_OK;
 }

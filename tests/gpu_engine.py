@@ -96,6 +96,22 @@ class GpuEngine:
                                    cv, n * self.model.conv_bytes)
         return st.cpu().numpy(), cv.cpu().numpy()
 
+    def gather_step(self, kv_first, kv_n, ssm_first, ssm_n, reqs, capacity_tokens):
+        """Both gathers in one launch -> (K [kv_n][cap][row], V, cu_seqlens, state [ssm_n][n][..], conv, error items)."""
+        r = np.ascontiguousarray(reqs, dtype=np.uint32)
+        row, n, cap = self.model.kv_row_bytes, max(len(r), 1), max(capacity_tokens, 1)
+        out_k = torch.zeros((kv_n, cap, row), dtype=torch.uint8, device=self.dev)
+        out_v = torch.zeros((kv_n, cap, row), dtype=torch.uint8, device=self.dev)
+        cu = torch.zeros(len(r) + 1, dtype=torch.int32, device=self.dev)
+        st = torch.zeros((ssm_n, n, self.model.state_bytes), dtype=torch.uint8, device=self.dev)
+        cv = torch.zeros((ssm_n, n, self.model.conv_bytes), dtype=torch.uint8, device=self.dev)
+        before = self.ctx.stats()["error_count"]
+        self.ctx.gather_step(self._dev(r), len(r), kv_first, kv_n, out_k, out_v, cap * row, capacity_tokens, cu,
+                             ssm_first, ssm_n, st, n * self.model.state_bytes, cv, n * self.model.conv_bytes)
+        bad = self.ctx.stats()["error_count"] - before
+        return (out_k.cpu().numpy(), out_v.cpu().numpy(), cu.cpu().numpy().view(np.uint32),
+                st.cpu().numpy(), cv.cpu().numpy(), bad)
+
     def scatter_kv(self, layer, reqs, tok_start, in_k, in_v) -> int:
         r = np.ascontiguousarray(reqs, dtype=np.uint32)
         before = self.ctx.stats()["error_count"]

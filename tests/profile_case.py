@@ -1,5 +1,5 @@
 """Small, self-contained launches of each kernel for profiling (a few GB on the device,
-a handful of launches): `python -m paper_2605_22416_b200.profile_case <case>`.
+a handful of launches): `python tests/profile_case.py <case>`.  Measurement tooling, not part of the library.
 
 Cases: ssm_gather, kv_gather (one layer per launch), ssm_gather_fused, kv_gather_fused (several
 layers per launch), relocate, step.  Every case builds a context through the
@@ -13,8 +13,13 @@ import argparse
 import numpy as np
 import torch
 
-from . import binding as B
-from . import workloads as W
+import sys
+from pathlib import Path
+
+sys.path.insert(0, str(Path(__file__).resolve().parent.parent))
+
+from paper_2605_22416_b200 import binding as B  # noqa: E402
+from paper_2605_22416_b200 import workloads as W  # noqa: E402
 
 
 def _dev(a):

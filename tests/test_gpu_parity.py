@@ -166,6 +166,18 @@ def test_random_shapes_and_policies(env, case):
                 assert e.scatter_ssm(layer, live, sb, cb) == 0
             gs, gc, gb = g.gather_ssm(layer, live)
             assert gb == 0 and np.array_equal(gs, sb) and np.array_equal(gc, cb)
+        # both gathers of all layers in one launch, on the held list (KV_ONLY slots are SSM error items)
+        fk, fv, fcu, fs, fc, fbad = g.gather_step(0, shape.n_attn_layers, 0, shape.n_ssm_layers, held, tot)
+        assert fbad == (len(held) - len(live)) * shape.n_ssm_layers
+        is_live = t["req_state"][held] == 1
+        for layer in range(shape.n_attn_layers):
+            ok, ov, ocu, _ = o.gather_kv(layer, held, tot)
+            assert np.array_equal(fcu, ocu) and np.array_equal(fk[layer, :tot], ok) and np.array_equal(fv[layer, :tot], ov)
+        for layer in range(shape.n_ssm_layers):
+            os_, oc, _ = o.gather_ssm(layer, held)
+            assert np.array_equal(fs[layer, :len(held)][is_live], os_[is_live])
+            assert np.array_equal(fc[layer, :len(held)][is_live], oc[is_live])
+        g.ctx.clear_error()
     assert g.stats()["error_code"] == 0
 
 
@@ -425,9 +437,6 @@ def test_full_size_configs(env, name, steps, over):
         assert s["relocated_blocks"] > 100
 
 
-_FULL_SCALE = 1_000_000 if os.environ.get("AVMP_FULL_SCALE") else 60_000
-
-
 @pytest.mark.parametrize("name,over,n_requests,max_steps", [
     ("short_uniform", dict(seed=0), None, None),
     ("short_uniform", dict(seed=1), None, None),
@@ -435,13 +444,13 @@ _FULL_SCALE = 1_000_000 if os.environ.get("AVMP_FULL_SCALE") else 60_000
     ("mixed_long", dict(migration_batch_size=16), None, None),
     ("mixed_long", dict(migration_batch_size=64), None, None),
     ("agentic_burst", {}, None, 20_000),
-    ("scale", {}, _FULL_SCALE, None),
+    ("scale", {}, None, None),
     ("scale", dict(split=0.9, migration_enabled=False), 30_000, None),
 ])
 def test_full_traces_allocator_only(env, name, over, n_requests, max_steps):
-    """The whole trace of every configuration (config 5: its first 60 000 requests unless
-    AVMP_FULL_SCALE is set), allocator only: every status of every step, the counters every 512
-    steps, every table at the end."""
+    """The whole trace of every configuration (config 5: all 1 000 000 requests, 3.8e8 operations in
+    370 000 steps; its static 0.9 partition on the first 30 000), allocator only: every status of every
+    step, the counters every 512 steps, every table at the end."""
     w = W.config(name, **over)
     g, o = _pair(env, w)
     d = W.ClosedLoopDriver(w, requests=W.make_requests(w, n_requests) if n_requests else None)
@@ -465,11 +474,13 @@ def test_full_traces_allocator_only(env, name, over, n_requests, max_steps):
 
 @pytest.mark.parametrize("split,enabled", [(0.5, True), (0.5, False), (0.9, False)])
 def test_scale_config(env, split, enabled):
-    """Config 5: 72-layer model, 120 GiB pool resident in HBM, step batch 1024."""
+    """Config 5: 72-layer model, 120 GiB pool resident in HBM, step batch 1024; payload on three
+    attention and three SSM layers (first, middle, last), gathers of the whole running batch on a
+    rotating pair of them against the payload function."""
     w = W.config("scale", split=split, migration_enabled=enabled)
-    s, seen, d = _closed_loop_parity(env, w, 80 if enabled else 50, with_store=False, kv_layers=[4],
-                                     ssm_layers=[31], table_every=25, gather_every=23, max_migration_checks=6)
-    assert seen["tokens"] > 0 and s["op_counter"] > 30_000
+    s, seen, d = _closed_loop_parity(env, w, 240 if enabled else 120, with_store=False, kv_layers=[0, 4, 8],
+                                     ssm_layers=[0, 31, 62], table_every=40, gather_every=47, max_migration_checks=4)
+    assert seen["tokens"] > (1_000_000 if enabled else 500_000) and s["op_counter"] > 100_000
 
 
 def test_sensitivity_sweep_cells_match_the_oracle(env):
@@ -942,3 +953,55 @@ def test_bytes_inside_a_unit_follow_the_documented_layout_on_gpu(env, shape):
 
     assert check_unit_layout(w, o, read_units_o) == seen
     env["same"](g, o, w, "layout run")
+
+
+@pytest.mark.parametrize("n_list", [0, 9, 1024, 1500])
+def test_step_gather_in_one_launch(env, n_list):
+    """avmp_gather_step: every attention layer and every SSM layer of a request list in one launch equals the
+    oracle's single-layer gathers (and the multi-layer entry points); lists on both sides of the 1024-entry
+    plan switch, with empty slots in between; layer sub-ranges; a buffer one row too small."""
+    w = W.config("pr1", pool_bytes=64 * W.MiB, max_requests=1536, concurrency=16, min_rebalance_interval_ops=50,
+                 migration_batch_size=6, n_requests=120)
+    g, o = _pair(env, w, with_store=True)
+    h = PayloadHarness(w, [g, o])
+    d = W.ClosedLoopDriver(w)
+
+    def step(ops):
+        so = o.step(ops)
+        assert np.array_equal(g.step(ops), so)
+        return so
+
+    W.record_trace(w, step, max_steps=120, driver=d, on_step=lambda d, a, b: h.apply_writes(d.writes))
+    assert g.stats()["n_rebalance"] > 0
+    m = w.model
+    run = d.running_slots.astype(np.uint32)
+    assert len(run) >= 9
+    reqs = np.resize(run[:9], n_list).astype(np.uint32)
+    if n_list > 9:
+        reqs[4::53] = 1400                                       # empty slots
+    n_empty = int((reqs == 1400).sum())
+    tot = int(o.tables()["req_len"][reqs].sum())
+
+    def check(kv_first, kv_n, ssm_first, ssm_n, cap):
+        fk, fv, fcu, fs, fc, bad = g.gather_step(kv_first, kv_n, ssm_first, ssm_n, reqs, cap)
+        want_bad = 0
+        for l in range(kv_n):
+            ok, ov, ocu, ob = o.gather_kv(kv_first + l, reqs, cap)
+            want_bad += ob if l == 0 else 0                      # the KV plan reports a list's bad items once
+            assert np.array_equal(fcu, ocu)
+            assert np.array_equal(fk[l, :cap], ok) and np.array_equal(fv[l, :cap], ov), (l, cap)
+        for l in range(ssm_n):
+            os_, oc, ob = o.gather_ssm(ssm_first + l, reqs)
+            want_bad += ob
+            assert np.array_equal(fs[l, :len(reqs)], os_) and np.array_equal(fc[l, :len(reqs)], oc), l
+        assert bad == want_bad and want_bad == n_empty * (1 + ssm_n) + (1 if cap < tot else 0)
+        return fk, fv, fs, fc
+
+    fk, fv, fs, fc = check(0, m.n_attn_layers, 0, m.n_ssm_layers, tot)
+    if n_list:
+        gk, gv, _ = g.gather_kv_layers(0, m.n_attn_layers, reqs, tot)
+        gs, gc = g.gather_ssm_layers(0, m.n_ssm_layers, reqs)
+        assert np.array_equal(fk, gk) and np.array_equal(fv, gv) and np.array_equal(fs, gs) and np.array_equal(fc, gc)
+        check(1, 2, 7, 3, tot)
+        check(3, 1, 11, 1, tot - 1)                               # the last request does not fit: it copies nothing
+    g.ctx.clear_error()
