@@ -239,7 +239,7 @@ def measure(w: W.Workload, dev, *, steps: int, warmup: int, warm_steps: int, ask
     # when the batch buffers of all layers fit, a step's payload moves in ONE launch (avmp_gather_step)
     one_launch = len(kv_groups) == 1 and len(ssm_groups) == 1
 
-    def full_step(c, r, marks=None, per_layer=False, fused=False):
+    def full_step(c, r, marks=None, per_layer=False, fused=False, separate_calls=False):
         """One engine step.  marks: one event pair per kernel class (allocator, KV, SSM).
         per_layer: one launch per layer instead of one launch per group of layers.
         fused: both gathers of all layers in one launch (the KV mark then coincides with the allocator mark)."""
@@ -249,8 +249,11 @@ def measure(w: W.Workload, dev, *, steps: int, warmup: int, warm_steps: int, ask
         e = [ev() for _ in range(4)] if marks is not None else None
         if e:
             e[0].record(stream)
-        c.step(r["d_ops"], n_ops, d_status, sid)
-        c.translate(r["d_handles"], len(r["handles"]), d_pool, d_off, d_aoff, sid)
+        if separate_calls:
+            c.step(r["d_ops"], n_ops, d_status, sid)
+            c.translate(r["d_handles"], len(r["handles"]), d_pool, d_off, d_aoff, sid)
+        else:       # the same two operations, the translation riding on the step's relocation-copy launch
+            c.step_translate(r["d_ops"], n_ops, d_status, r["d_handles"], len(r["handles"]), d_pool, d_off, d_aoff, sid)
         if e:
             e[1].record(stream)
         if fused:
@@ -323,7 +326,7 @@ def measure(w: W.Workload, dev, *, steps: int, warmup: int, warm_steps: int, ask
         c = fresh_context()
         marks = []
         for r in timed:
-            full_step(c, r, marks, per_layer=per_layer, fused=fused)
+            full_step(c, r, marks, per_layer=per_layer, fused=fused, separate_calls=per_layer)
         torch.cuda.synchronize(dev)
         st = c.stats()
         c.close()
@@ -403,6 +406,7 @@ def class_figures(res: dict, m: W.ModelShape, peak: float) -> dict:
     out = {"ssm_gbs": ssm_launch_bytes / (ssm_ms * 1e-3) / 1e9, "ssm_launch_ms": ssm_ms, "ssm_launch_bytes": ssm_launch_bytes,
            "kv_gbs": kv_launch_bytes / (kv_ms * 1e-3) / 1e9, "kv_launch_ms": kv_ms, "kv_launch_bytes": kv_launch_bytes,
            "allocator_us_per_step": step_ms * 1e3, "allocator_ops_per_s": res["n_ops"] / (sum(per["step"]) * 1e-3),
+           "allocator_us_per_step_separate_calls": float(np.mean(res["per_l"]["step"])) * 1e3 if res["per_l"] is not None else None,
            "unit_allocs_frees_per_s": res["units"] / (sum(per["step"]) * 1e-3)}
     if res["per_f"] is not None:
         ms = float(np.mean([a + b for a, b in zip(res["per_f"]["kv"], res["per_f"]["ssm"])]))   # kv mark is empty
@@ -465,9 +469,11 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
                                              "note": "same window, avmp_gather_kv once per layer, back to back"},
                          "allocator_ops_per_s": f["allocator_ops_per_s"] * (world if world > 1 else 1),
                          "allocator_us_per_step": f["allocator_us_per_step"],
+                         "allocator_us_per_step_separate_calls": f["allocator_us_per_step_separate_calls"],
                          "unit_allocs_frees_per_s": f["unit_allocs_frees_per_s"],
-                         "allocator_note": "avmp_step + avmp_translate of every live handle of the batch, CUDA events "
-                                           "around the two calls, rank 0's timing; units = KV pages + SSM blocks allocated "
+                         "allocator_note": "avmp_step_translate (allocator step + translate of every live handle of the batch; "
+                                           "the translation rides on the step's relocation-copy launch), CUDA events around "
+                                           "the call, rank 0's timing; separate_calls = avmp_step then avmp_translate; units = KV pages + SSM blocks allocated "
                                            "or freed, counted from the request slots' net change per step"}},
         "e2e": {"value": sums[0] / (e2e_ms_g * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms_g / K,
                 "h2d_bytes_per_step": sums[5] / K / world, "d2h_bytes_per_step": sums[6] / K / world,

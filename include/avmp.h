@@ -210,6 +210,14 @@ AVMP_API int avmp_destroy(avmp_ctx *ctx);
  * Stream-ordered, no host synchronisation.  n_ops == 0 is a no-op. */
 AVMP_API int avmp_step(avmp_ctx *ctx, const avmp_op *d_ops, uint32_t n_ops, uint32_t *d_status, void *stream);
 
+/* avmp_step followed by avmp_translate of d_handles against the tables that step leaves (Sections 3.1-3.2
+ * and Figure 1), with the translation riding on the step's relocation-copy launch: two launches per engine
+ * step instead of three, which is most of what the allocator part of a step costs.  Results are exactly those
+ * of the two calls made one after the other.  n_handles == 0 is avmp_step; n_ops == 0 is avmp_translate. */
+AVMP_API int avmp_step_translate(avmp_ctx *ctx, const avmp_op *d_ops, uint32_t n_ops, uint32_t *d_status,
+                                 const uint32_t *d_handles, uint32_t n_handles, uint32_t *d_pool, uint64_t *d_offset,
+                                 uint64_t *d_arena_offset, void *stream);
+
 /* Same step, with the batch length read from device memory when the kernel runs (*d_n_ops, clamped
  * to max_ops): for batches that another kernel builds, so that a serving loop needs no host round
  * trip per step.  max_ops bounds the work the host queues (the number of migration rounds). */

@@ -93,6 +93,7 @@ def _load():
                                   C.c_uint32, C.POINTER(avmp_options), vp, C.c_size_t, vp]),
         "avmp_destroy": (C.c_int, [vp]),
         "avmp_step": (C.c_int, [vp, vp, C.c_uint32, vp, vp]),
+        "avmp_step_translate": (C.c_int, [vp, vp, C.c_uint32, vp, vp, C.c_uint32, vp, vp, vp, vp]),
         "avmp_step_host": (C.c_int, [vp, vp, C.c_uint32, vp, vp]),
         "avmp_step_indirect": (C.c_int, [vp, vp, vp, C.c_uint32, vp, vp]),
         "avmp_driver_workspace_bytes": (C.c_size_t, [C.c_uint32]),
@@ -200,6 +201,12 @@ def avmp_destroy(ctx):
 
 def avmp_step(ctx, d_ops, n_ops, d_status, stream=None):
     _check(lib.avmp_step(ctx, _ptr(d_ops), n_ops, _ptr(d_status), _stream(stream)), "avmp_step")
+
+
+def avmp_step_translate(ctx, d_ops, n_ops, d_status, d_handles, n_handles, d_pool, d_offset, d_arena_offset=None,
+                        stream=None):
+    _check(lib.avmp_step_translate(ctx, _ptr(d_ops), n_ops, _ptr(d_status), _ptr(d_handles), n_handles, _ptr(d_pool),
+                                   _ptr(d_offset), _ptr(d_arena_offset), _stream(stream)), "avmp_step_translate")
 
 
 def avmp_step_host(ctx, h_ops, n_ops, h_status, stream=None):
@@ -476,6 +483,11 @@ class Context:
 
     def step(self, d_ops, n_ops, d_status, stream=None):
         avmp_step(self.handle, d_ops, n_ops, d_status, stream)
+
+    def step_translate(self, d_ops, n_ops, d_status, d_handles, n_handles, d_pool, d_offset, d_arena_offset=None,
+                       stream=None):
+        avmp_step_translate(self.handle, d_ops, n_ops, d_status, d_handles, n_handles, d_pool, d_offset,
+                            d_arena_offset, stream)
 
     def step_host(self, h_ops, n_ops, h_status, stream=None):
         avmp_step_host(self.handle, h_ops, n_ops, h_status, stream)

@@ -285,8 +285,16 @@ int avmp_destroy(avmp_ctx *c)
     return AVMP_OK;
 }
 
+// A handle list to translate against the tables the step leaves (may be empty).
+struct TranslateArgs {
+    const uint32_t *h = nullptr;
+    uint32_t n = 0;
+    uint32_t *pool = nullptr;
+    unsigned long long *off = nullptr, *aoff = nullptr;
+};
+
 static int step_rounds(avmp_ctx *c, const avmp_op *d_ops, uint32_t n_ops, const uint32_t *d_n_ops,
-                       uint32_t *d_status, void *stream)
+                       uint32_t *d_status, void *stream, const TranslateArgs &tr = TranslateArgs())
 {
     // Section 3.2 throttle: migrations are >= min_interval logical ops apart, so a batch of n ops
     // holds at most (n - 1) / min_interval + 1 of them; one launch performs at most one.
@@ -297,9 +305,17 @@ static int step_rounds(avmp_ctx *c, const avmp_op *d_ops, uint32_t n_ops, const 
         if (launch_step(c->g, d_ops, n_ops, d_n_ops, d_status, r == 0, S(stream)) != cudaSuccess) return AVMP_ECUDA;
         c->launches += 1;
         if (c->opt.migration_enabled) {
-            if (launch_relocate(c->g, L(c, stream)) != cudaSuccess) return AVMP_ECUDA;
+            // the last round's copy launch also carries the translation: two launches per step, not three
+            const cudaError_t e = (tr.n && r + 1 == rounds)
+                                      ? launch_relocate_translate(c->g, tr.h, tr.n, tr.pool, tr.off, tr.aoff, L(c, stream))
+                                      : launch_relocate(c->g, L(c, stream));
+            if (e != cudaSuccess) return AVMP_ECUDA;
             c->launches += 1;
         }
+    }
+    if (tr.n && !c->opt.migration_enabled) {
+        if (launch_translate(c->g, tr.h, tr.n, tr.pool, tr.off, tr.aoff, L(c, stream)) != cudaSuccess) return AVMP_ECUDA;
+        c->launches += 1;
     }
     return AVMP_OK;
 }
@@ -310,6 +326,19 @@ int avmp_step(avmp_ctx *c, const avmp_op *d_ops, uint32_t n_ops, uint32_t *d_sta
     if (n_ops == 0) return AVMP_OK;
     if (!d_ops || !d_status || ((uintptr_t)d_ops & 3) || ((uintptr_t)d_status & 3)) return AVMP_EINVAL;
     return step_rounds(c, d_ops, n_ops, nullptr, d_status, stream);
+}
+
+int avmp_step_translate(avmp_ctx *c, const avmp_op *d_ops, uint32_t n_ops, uint32_t *d_status, const uint32_t *d_handles,
+                        uint32_t n_handles, uint32_t *d_pool, uint64_t *d_offset, uint64_t *d_arena_offset, void *stream)
+{
+    if (!c) return AVMP_EINVAL;
+    if (n_handles && (!d_handles || !d_pool || !d_offset)) return AVMP_EINVAL;
+    if (n_ops == 0) return avmp_translate(c, d_handles, n_handles, d_pool, d_offset, d_arena_offset, stream);
+    if (!d_ops || !d_status || ((uintptr_t)d_ops & 3) || ((uintptr_t)d_status & 3)) return AVMP_EINVAL;
+    TranslateArgs tr;
+    tr.h = d_handles; tr.n = n_handles; tr.pool = d_pool;
+    tr.off = (unsigned long long *)d_offset; tr.aoff = (unsigned long long *)d_arena_offset;
+    return step_rounds(c, d_ops, n_ops, nullptr, d_status, stream, tr);
 }
 
 int avmp_step_indirect(avmp_ctx *c, const avmp_op *d_ops, const uint32_t *d_n_ops, uint32_t max_ops,

@@ -55,6 +55,7 @@ template <bool SCATTER>
 struct SsmPieces {
     static constexpr bool kTimed = false;
     static constexpr bool kPlans = false;
+    static constexpr bool kTail = false;
     uint32_t layer0, n_layers, n, ps, per;
     const uint32_t *reqs;
     uint8_t *buf_state, *buf_conv;
@@ -96,6 +97,7 @@ struct SsmPieces {
 struct RelocPieces {
     static constexpr bool kTimed = true;     // the copy stamps the device clock: migration time is a metric
     static constexpr bool kPlans = false;
+    static constexpr bool kTail = false;
     __device__ unsigned long long total(const Geom &g) const
     {
         const unsigned long long U = g.U[g.st->reloc_pool];
@@ -111,6 +113,39 @@ struct RelocPieces {
         // dst < new capacity <= src: the two units never overlap
         return Piece{unit_ptr(g, pool, g.reloc_src[k]) + o, unit_ptr(g, pool, g.reloc_dst[k]) + o,
                      (uint32_t)min((unsigned long long)kStage, U - o)};
+    }
+};
+
+// a10 for one handle: pool tag, offset inside that store, offset inside the arena.
+__device__ __forceinline__ void translate_one(const Geom &g, uint32_t hv, uint32_t i, uint32_t *__restrict__ pool,
+                                              unsigned long long *__restrict__ off, unsigned long long *__restrict__ aoff)
+{
+    const uint32_t p = hv >> 31, vid = hv & 0x7FFFFFFFu;
+    uint32_t slot = kInvalid;
+    if (hv != kInvalid && vid < g.V[p]) slot = g.VT[p][vid];
+    if (slot == kInvalid) {
+        pool[i] = kInvalid; off[i] = kNone64;
+        if (aoff) aoff[i] = kNone64;
+        record_error(g.st, AVMP_DEV_BAD_HANDLE);
+    } else {
+        pool[i] = p; off[i] = (unsigned long long)slot * g.U[p];
+        if (aoff) aoff[i] = (unsigned long long)(unit_ptr(g, p, slot) - g.arena);
+    }
+}
+
+// a7 + a10 in one launch: the relocation copy of a step, and the translation of a handle list against the
+// tables that step left (the page table is remapped by the step kernel itself, so the look-ups do not
+// depend on the copy).  Saves the third launch of an engine step's allocator part.
+struct RelocTranslate : RelocPieces {
+    static constexpr bool kTail = true;
+    const uint32_t *h;
+    uint32_t n;
+    uint32_t *pool;
+    unsigned long long *off, *aoff;
+    __device__ void tail(const Geom &g) const
+    {
+        for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
+            translate_one(g, h[i], i, pool, off, aoff);
     }
 };
 
@@ -147,6 +182,7 @@ template <bool SCATTER>
 struct KvPieces {
     static constexpr bool kTimed = false;
     static constexpr bool kPlans = true;
+    static constexpr bool kTail = false;
     uint32_t layer0, n_layers, n, subs;
     const uint32_t *reqs, *tok_start;
     uint8_t *buf_k, *buf_v;
@@ -261,6 +297,7 @@ struct KvPieces {
 struct StepPieces {
     static constexpr bool kTimed = false;
     static constexpr bool kPlans = true;
+    static constexpr bool kTail = false;
     KvPieces<false> kv;
     SsmPieces<false> ssm;
     __device__ void plan(const Geom &g, uint32_t *buf, unsigned long long *tmp) { kv.plan(g, buf, tmp); }
@@ -404,6 +441,7 @@ __global__ void __launch_bounds__(kBulkThreads, kBulkCtasPerSm) stream_bulk_kern
     pdl_prologue();
     __syncthreads();
     F f = f_in;
+    if constexpr (F::kTail) f.tail(g);
     if constexpr (F::kPlans) {
         __shared__ uint32_t plan_buf[kPlanWords];
         __shared__ unsigned long long plan_tmp[32];
@@ -465,6 +503,7 @@ __global__ void __launch_bounds__(kGenThreads) stream_generic_kernel(const Geom 
     const int lane = threadIdx.x & 31;
     pdl_prologue();
     F f = f_in;
+    if constexpr (F::kTail) f.tail(g);
     if constexpr (F::kPlans) {
         __shared__ uint32_t plan_buf[kPlanWords];
         __shared__ unsigned long long plan_tmp[32];
@@ -514,19 +553,8 @@ __global__ void translate_kernel(const Geom g, const uint32_t *__restrict__ h, u
                                  unsigned long long *__restrict__ aoff)
 {
     pdl_prologue();
-    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
-        const uint32_t hv = h[i], p = hv >> 31, vid = hv & 0x7FFFFFFFu;
-        uint32_t slot = kInvalid;
-        if (hv != kInvalid && vid < g.V[p]) slot = g.VT[p][vid];
-        if (slot == kInvalid) {
-            pool[i] = kInvalid; off[i] = kNone64;
-            if (aoff) aoff[i] = kNone64;
-            record_error(g.st, AVMP_DEV_BAD_HANDLE);
-        } else {
-            pool[i] = p; off[i] = (unsigned long long)slot * g.U[p];
-            if (aoff) aoff[i] = (unsigned long long)(unit_ptr(g, p, slot) - g.arena);
-        }
-    }
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
+        translate_one(g, h[i], i, pool, off, aoff);
 }
 
 // ---- a11 plan: request list -> row prefix sums (cu_seqlens) and piece prefix sums --------
@@ -566,6 +594,14 @@ kv_plan_kernel(const Geom g, const uint32_t *__restrict__ reqs, const uint32_t *
 cudaError_t launch_relocate(const Geom &g, const Launch &l)
 {
     return launch_stream(g, RelocPieces{}, mult16(g.U[0]) && mult16(g.U[1]) && mult16(g.P_al), l);
+}
+
+cudaError_t launch_relocate_translate(const Geom &g, const uint32_t *h, uint32_t n, uint32_t *pool,
+                                      unsigned long long *off, unsigned long long *aoff, const Launch &l)
+{
+    RelocTranslate f;
+    f.h = h; f.n = n; f.pool = pool; f.off = off; f.aoff = aoff;
+    return launch_stream(g, f, mult16(g.U[0]) && mult16(g.U[1]) && mult16(g.P_al), l);
 }
 
 cudaError_t launch_translate(const Geom &g, const uint32_t *h, uint32_t n, uint32_t *pool,

@@ -167,6 +167,8 @@ cudaError_t launch_init(const Geom &g, const DevState &init, cudaStream_t s);
 cudaError_t launch_step(const Geom &g, const avmp_op *d_ops, uint32_t n_ops, const uint32_t *d_n_ops,
                         uint32_t *d_status, int first_round, cudaStream_t s);
 cudaError_t launch_relocate(const Geom &g, const Launch &l);
+cudaError_t launch_relocate_translate(const Geom &g, const uint32_t *h, uint32_t n, uint32_t *pool,
+                                      unsigned long long *off, unsigned long long *aoff, const Launch &l);
 cudaError_t launch_translate(const Geom &g, const uint32_t *h, uint32_t n, uint32_t *pool,
                              unsigned long long *off, unsigned long long *aoff, const Launch &l);
 cudaError_t launch_kv(const Geom &g, bool scatter, uint32_t layer0, uint32_t n_layers, const uint32_t *reqs,

@@ -1,5 +1,17 @@
 // The allocator update of one batch as a device function over one CTA (see avmp_step.cu for the
 // method): shared by the plain step kernel and by the fused on-device loop.
+//
+// The path is latency-bound: one CTA, a chain of dependent global round trips with block barriers
+// between them.  What keeps the chain short:
+//   * the free counts live in registers (every thread holds the same copy and updates it from
+//     block-wide totals), so no phase ends with "thread 0 updates, everyone waits";
+//   * scans and minima cost one barrier each (double-buffered partials, every thread sums the few
+//     warp totals itself);
+//   * a window whose ops come as FINISH*, EXTEND*, ADMIT* with ascending slots inside each kind --
+//     the shape every engine step has -- is recognised with one ballot per warp: its two runs are
+//     known at once, no same-slot table and no run search is needed;
+//   * an alloc run whose total demand fits is committed in one pass; only a shortage takes the
+//     search for the first failing op and the CapacityError handler.
 #pragma once
 
 #include "avmp_dev.cuh"
@@ -24,9 +36,8 @@ struct Scalars {
     unsigned long long mig_waste;
 };
 
-// NT = threads of the planning CTA = ops per window.  Small batches run with a small CTA: the
-// kernel is a chain of some forty block barriers, and a barrier over 8 warps costs a fraction of
-// one over 32.
+// NT = threads of the planning CTA = ops per window.  Small batches run with a small CTA: a barrier
+// over 8 warps costs a fraction of one over 32.
 template <int NT>
 struct Shared {
     static constexpr uint32_t kHash = 2 * NT;     // open-addressing table for same-slot detection
@@ -34,10 +45,54 @@ struct Shared {
     uint32_t req[NT], base[NT];
     uint32_t hkey[kHash], hval[kHash];
     uint8_t dir[NT];
-    unsigned long long tmp64[32];
+    unsigned long long scan_part[2][32];          // one-barrier scans: warp totals, double-buffered
+    uint32_t min_part[2][32];
+    unsigned long long tmp64[32];                 // the handler's and the run search's own partials
     uint32_t tmp32[32];
+    uint32_t w_shape[32];                         // per warp: window-shape flag and number of FINISH ops
+    uint32_t start;                               // first op of this launch (multi-round steps)
+    uint32_t n_inv;                               // ops rejected in this launch
     Scalars sc;
 };
+
+// Inclusive scan over the block with ONE barrier: every thread adds up the warp totals before its own
+// warp.  `flip` (the same in every thread) alternates the two partial buffers, so the next scan may
+// write while slow threads still read this one's partials.
+template <int NT>
+__device__ __forceinline__ unsigned long long scan1(unsigned long long v, unsigned long long (*part)[32], uint32_t &flip,
+                                                    unsigned long long *total)
+{
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    unsigned long long *t = part[flip & 1u];
+    flip ^= 1u;
+    v = warp_incl_scan(v);
+    if (lane == 31) t[wid] = v;
+    __syncthreads();
+    unsigned long long off = 0, tot = 0;
+#pragma unroll
+    for (int w = 0; w < NT / 32; ++w) {
+        const unsigned long long x = t[w];
+        tot += x;
+        if (w < wid) off += x;
+    }
+    *total = tot;
+    return v + off;
+}
+
+template <int NT>
+__device__ __forceinline__ uint32_t min1(uint32_t v, uint32_t (*part)[32], uint32_t &flip)
+{
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    uint32_t *t = part[flip & 1u];
+    flip ^= 1u;
+    v = __reduce_min_sync(0xFFFFFFFFu, v);
+    if (lane == 0) t[wid] = v;
+    __syncthreads();
+    uint32_t m = INF;
+#pragma unroll
+    for (int w = 0; w < NT / 32; ++w) m = min(m, t[w]);
+    return m;
+}
 
 __device__ __forceinline__ bool would_migrate(const Geom &g, const Scalars &sc, int X, unsigned long long counter)
 {
@@ -156,15 +211,15 @@ __device__ void capacity_error(const Geom &g, Shared<NT> &sh, int X, unsigned lo
     __syncthreads();
 }
 
-// Pop units for the ops [lo, hi) of the current alloc scan (none of them fails).
+// Pop units for the ops [lo, hi) of the current alloc scan (none of them fails): unit u of the run
+// takes stack entry (top - 1 - u).  fk / vk / fs / vs are the stack heights before the run.
 template <int NT>
-__device__ __forceinline__ void commit_allocs(const Geom &g, Shared<NT> &sh, uint32_t lo, uint32_t hi)
+__device__ __forceinline__ void pop_units(const Geom &g, Shared<NT> &sh, uint32_t lo, uint32_t hi,
+                                          uint32_t fk, uint32_t vk, uint32_t fs, uint32_t vs, uint32_t &Tk, uint32_t &Ts)
 {
-    Scalars &sc = sh.sc;
     const int tid = threadIdx.x;
     const uint32_t bk = sh.excl_k[lo], bs = sh.excl_s[lo];
-    const uint32_t Tk = sh.excl_k[hi] - bk, Ts = sh.excl_s[hi] - bs;
-    const uint32_t fk = sc.nfree[0], vk = sc.nvfree[0], fs = sc.nfree[1], vs = sc.nvfree[1];
+    Tk = sh.excl_k[hi] - bk; Ts = sh.excl_s[hi] - bs;
     for (uint32_t u = tid; u < Tk; u += NT) {
         const uint32_t idx = find_owner(sh.excl_k, lo, hi, bk, u);
         const uint32_t j = u - (sh.excl_k[idx] - bk);
@@ -181,8 +236,17 @@ __device__ __forceinline__ void commit_allocs(const Geom &g, Shared<NT> &sh, uin
         g.OW[1][slot] = vid;
         g.r_ssm[(unsigned long long)sh.req[idx] * g.ns + j] = 0x80000000u | vid;
     }
+}
+
+// The same with the heights in shared memory (the shortage path keeps them there for the handler).
+template <int NT>
+__device__ __forceinline__ void commit_allocs(const Geom &g, Shared<NT> &sh, uint32_t lo, uint32_t hi)
+{
+    Scalars &sc = sh.sc;
+    uint32_t Tk, Ts;
+    pop_units<NT>(g, sh, lo, hi, sc.nfree[0], sc.nvfree[0], sc.nfree[1], sc.nvfree[1], Tk, Ts);
     __syncthreads();
-    if (tid == 0) {
+    if (threadIdx.x == 0) {
         sc.nfree[0] -= Tk; sc.nvfree[0] -= Tk;
         sc.nfree[1] -= Ts; sc.nvfree[1] -= Ts;
     }
@@ -197,43 +261,70 @@ __device__ void step_body(const Geom &g, Shared<NT> &sh, const avmp_op *__restri
 {
     constexpr uint32_t kHash = Shared<NT>::kHash;
     Scalars &sc = sh.sc;
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     DevState *ds = g.st;
+    uint32_t flip_s = 0, flip_m = 0;                // buffer toggles of scan1 / min1, the same in every thread
 
+    // The first window's ops are fetched while thread 0 fetches the counters (first round: the batch
+    // starts at op 0; later rounds must learn where the last one stopped).
+    uint32_t pre_w0 = 0, pre_w1 = 0, pre_w2 = 0, pre_pw0 = 0, pre_pw1 = 0;
+    const bool preloaded = first_round != 0;
+    if (preloaded && (uint32_t)tid < n_ops) {
+        const uint32_t *w = reinterpret_cast<const uint32_t *>(ops + tid);
+        pre_w0 = w[0]; pre_w1 = w[1]; pre_w2 = w[2];
+        if (lane == 0 && tid > 0) { pre_pw0 = w[-3]; pre_pw1 = w[-2]; }     // the op before this warp's first
+    }
     if (tid == 0) {
-        sc.last = ds->last_rebalance_op; sc.n_oom = ds->n_oom; sc.n_ce = ds->n_capacity_error;
-        sc.n_reb = ds->n_rebalance; sc.migrated = ds->migrated_bytes; sc.wasted = ds->wasted_bytes;
-        sc.reloc_blocks = ds->relocated_blocks; sc.reloc_bytes = ds->relocated_bytes;
-        sc.gap = ds->gap_bytes; sc.n_invalid = ds->n_invalid; sc.counter_base = ds->op_counter;
+        const unsigned long long a0 = ds->last_rebalance_op, a1 = ds->n_oom, a2 = ds->n_capacity_error, a3 = ds->n_rebalance,
+                                 a4 = ds->migrated_bytes, a5 = ds->wasted_bytes, a6 = ds->relocated_blocks,
+                                 a7 = ds->relocated_bytes, a8 = ds->gap_bytes, a9 = ds->n_invalid, a10 = ds->op_counter;
+        const uint32_t c0 = ds->cap[0], c1 = ds->cap[1], f0 = ds->n_free[0], f1 = ds->n_free[1], v0 = ds->n_vfree[0],
+                       v1 = ds->n_vfree[1], fsm = ds->fsm, pend = ds->reloc_pending, res = first_round ? 0u : ds->resume_idx;
+        sc.last = a0; sc.n_oom = a1; sc.n_ce = a2; sc.n_reb = a3; sc.migrated = a4; sc.wasted = a5;
+        sc.reloc_blocks = a6; sc.reloc_bytes = a7; sc.gap = a8; sc.n_invalid = a9; sc.counter_base = a10;
         sc.t_start = clock64(); sc.cyc_oom = 0; sc.cyc_mig = 0;
-        for (int p = 0; p < 2; ++p) { sc.cap[p] = ds->cap[p]; sc.nfree[p] = ds->n_free[p]; sc.nvfree[p] = ds->n_vfree[p]; }
-        sc.fsm = ds->fsm;
-        if (ds->reloc_pending) {            // fold the last relocation copy's duration into the total
-            if (ds->reloc_t1 > ds->reloc_t0) ds->reloc_ns_total += ds->reloc_t1 - ds->reloc_t0;
+        sc.cap[0] = c0; sc.cap[1] = c1; sc.nfree[0] = f0; sc.nfree[1] = f1; sc.nvfree[0] = v0; sc.nvfree[1] = v1;
+        sc.fsm = fsm;
+        if (pend) {                         // fold the last relocation copy's duration into the total
+            const unsigned long long t0 = ds->reloc_t0, t1 = ds->reloc_t1;
+            if (t1 > t0) ds->reloc_ns_total += t1 - t0;
             ds->reloc_pending = 0;
         }
         sc.migs_done = 0; sc.abort = 0; sc.abort_idx = 0; sc.n_reloc = 0; sc.reloc_pool = 0;
         sc.mig = 0;
-        sh.excl_k[0] = first_round ? 0u : ds->resume_idx;    // borrow a slot to broadcast the start
+        sh.start = res;
+        sh.n_inv = 0;
     }
-    __syncthreads();
-    const uint32_t start = sh.excl_k[0];
-    __syncthreads();
-    if (start >= n_ops) {           // an earlier round finished the batch
+    uint32_t start = 0;
+    if (!preloaded) {
+        __syncthreads();
+        start = sh.start;
+    }
+    if (start >= n_ops) {               // an earlier round finished the batch (or the batch is empty)
         if (tid == 0) ds->n_reloc = 0;
         return;
     }
+    // free counts: registers, the same in every thread (filled after the first window's barrier)
+    uint32_t nf0 = 0, nv0 = 0, nf1 = 0, nv1 = 0;
+    bool have_counts = false;
 
     uint32_t done_upto = n_ops;     // ops [start, done_upto) are applied when the launch ends
+    bool aborted = false;
     for (uint32_t w0 = start; w0 < n_ops; w0 += NT) {
         const uint32_t wn = min((uint32_t)NT, n_ops - w0);
         // ---- decode (a1) ----
         uint32_t kind = 0, flags = 0, req = 0, tokens = 0, st = ST_PENDING;
+        uint32_t prev_word0 = 0, prev_req = 0;
         uint8_t dir = DIR_NONE;
-        if (tid < wn) {
-            const uint32_t *w = reinterpret_cast<const uint32_t *>(ops + (w0 + tid));
-            const uint32_t w0_ = w[0];
-            kind = w0_ & 0xFFu; flags = (w0_ >> 8) & 0xFFu; req = w[1]; tokens = w[2];
+        if (tid < (int)wn) {
+            uint32_t w0_, w1_, w2_;
+            if (preloaded && w0 == 0) { w0_ = pre_w0; w1_ = pre_w1; w2_ = pre_w2; prev_word0 = pre_pw0; prev_req = pre_pw1; }
+            else {
+                const uint32_t *w = reinterpret_cast<const uint32_t *>(ops + (w0 + tid));
+                w0_ = w[0]; w1_ = w[1]; w2_ = w[2];
+                if (lane == 0 && tid > 0) { prev_word0 = w[-3]; prev_req = w[-2]; }
+            }
+            kind = w0_ & 0xFFu; flags = (w0_ >> 8) & 0xFFu; req = w1_; tokens = w2_;
             dir = DIR_NOP;
             if (kind != AVMP_OP_ADMIT && kind != AVMP_OP_EXTEND && kind != AVMP_OP_FINISH) st = AVMP_ST_BAD_ARG;
             else if (req >= g.R) st = AVMP_ST_BAD_REQ;
@@ -246,36 +337,90 @@ __device__ void step_body(const Geom &g, Shared<NT> &sh, const avmp_op *__restri
         // appears earlier in the window read it again when their run starts
         uint32_t pf_state = 0, pf_len = 0, pf_np = 0;
         if (dir >= DIR_ALLOC) { pf_state = g.r_state[req]; pf_len = g.r_len[req]; pf_np = g.r_npages[req]; }
-        // ---- same-slot dependencies inside the window: shared-memory hash, slot -> first op ----
-        sh.hkey[tid] = INF; sh.hkey[tid + NT] = INF;
-        sh.hval[tid] = INF; sh.hval[tid + NT] = INF;
-        __syncthreads();
-        uint32_t hs = 0;
-        if (dir >= DIR_ALLOC) {
-            hs = (req * 2654435761u) & (kHash - 1u);
-            while (true) {
-                const uint32_t old = atomicCAS(&sh.hkey[hs], INF, req);
-                if (old == INF || old == req) break;
-                hs = (hs + 1u) & (kHash - 1u);
+
+        // ---- shape of the window: FINISH*, EXTEND*, ADMIT*, every op valid, slots ascending inside a kind ----
+        // rank: FINISH 0 < EXTEND 1 < ADMIT 2.  An op is in place if the op before it has a lower rank, or the same
+        // rank and a lower slot.  One ballot per warp; lane 0 compares with the op it fetched beside its own.
+        {
+            const uint32_t rank = kind == AVMP_OP_FINISH ? 0u : (kind == AVMP_OP_EXTEND ? 1u : 2u);
+            uint32_t p_rank = __shfl_up_sync(0xFFFFFFFFu, rank, 1), p_req = __shfl_up_sync(0xFFFFFFFFu, req, 1);
+            if (lane == 0) {
+                const uint32_t pk = prev_word0 & 0xFFu;
+                p_rank = pk == AVMP_OP_FINISH ? 0u : (pk == AVMP_OP_EXTEND ? 1u : 2u);
+                p_req = prev_req;
             }
-            atomicMin(&sh.hval[hs], (uint32_t)tid);
+            bool in_place = true;
+            if (tid < (int)wn) in_place = dir >= DIR_ALLOC && (tid == 0 || p_rank < rank || (p_rank == rank && p_req < req));
+            const uint32_t ok = __all_sync(0xFFFFFFFFu, in_place) ? 1u : 0u;
+            const uint32_t nfin = __popc(__ballot_sync(0xFFFFFFFFu, tid < (int)wn && dir == DIR_FREE));
+            if (lane == 0) sh.w_shape[wid] = (ok << 31) | nfin;
         }
-        __syncthreads();
-        const bool dupflag = dir >= DIR_ALLOC && sh.hval[hs] != (uint32_t)tid;
-        const int any_dup = __syncthreads_or(dupflag);
-        int prev_same = -1;
-        if (any_dup && dupflag)
-            for (int j = tid - 1; j >= 0; --j)
-                if (sh.dir[j] >= DIR_ALLOC && sh.req[j] == req) { prev_same = j; break; }
+        __syncthreads();                                    // B1: counters, dir / req, window shape
+        if (!have_counts) {
+            nf0 = sc.nfree[0]; nv0 = sc.nvfree[0]; nf1 = sc.nfree[1]; nv1 = sc.nvfree[1];
+            have_counts = true;
+        }
+        bool fast = true;
+        uint32_t nF = 0;
+#pragma unroll
+        for (int w = 0; w < NT / 32; ++w) {
+            const uint32_t x = sh.w_shape[w];
+            fast = fast && (x >> 31);
+            nF += x & 0x7FFFFFFFu;
+        }
+
+        // ---- same-slot dependencies inside the window ----
+        int prev_same = -1;        // >= 0: an earlier op of this window touches the same slot
+        if (fast) {
+            // Runs are [0, nF) and [nF, wn); slots are distinct inside each.  An alloc op only has to know
+            // whether a FINISH of this window released its slot (its prefetched record is then stale):
+            // the FINISH slots ascend, so a binary search answers that.
+            if (nF > 0 && tid >= (int)nF && tid < (int)wn) {
+                uint32_t lo = 0, hi = nF;
+                while (lo < hi) {
+                    const uint32_t mid = (lo + hi) >> 1;
+                    if (sh.req[mid] < req) lo = mid + 1; else hi = mid;
+                }
+                if (lo < nF && sh.req[lo] == req) prev_same = (int)lo;
+            }
+        } else {
+            // general windows: shared-memory hash, slot -> first op
+            sh.hkey[tid] = INF; sh.hkey[tid + NT] = INF;
+            sh.hval[tid] = INF; sh.hval[tid + NT] = INF;
+            __syncthreads();
+            uint32_t hs = 0;
+            if (dir >= DIR_ALLOC) {
+                hs = (req * 2654435761u) & (kHash - 1u);
+                while (true) {
+                    const uint32_t old = atomicCAS(&sh.hkey[hs], INF, req);
+                    if (old == INF || old == req) break;
+                    hs = (hs + 1u) & (kHash - 1u);
+                }
+                atomicMin(&sh.hval[hs], (uint32_t)tid);
+            }
+            __syncthreads();
+            const bool dupflag = dir >= DIR_ALLOC && sh.hval[hs] != (uint32_t)tid;
+            const int any_dup = __syncthreads_or(dupflag);
+            if (any_dup && dupflag)
+                for (int j = tid - 1; j >= 0; --j)
+                    if (sh.dir[j] >= DIR_ALLOC && sh.req[j] == req) { prev_same = j; break; }
+        }
 
         uint32_t cur = 0;
         while (cur < wn) {
-            const uint32_t first = block_min((tid >= (int)cur && dir >= DIR_ALLOC) ? (uint32_t)tid : INF, sh.tmp32);
-            if (first == INF) break;
-            const uint8_t rdir = sh.dir[first];
-            const bool stops = tid > (int)first && tid < (int)wn &&
-                               ((dir >= DIR_ALLOC && dir != rdir) || prev_same >= (int)cur);
-            const uint32_t end = block_min(stops ? (uint32_t)tid : wn, sh.tmp32);
+            uint32_t end;
+            uint8_t rdir;
+            if (fast) {
+                rdir = cur < nF ? DIR_FREE : DIR_ALLOC;
+                end = cur < nF ? nF : wn;
+            } else {
+                const uint32_t first = block_min((tid >= (int)cur && dir >= DIR_ALLOC) ? (uint32_t)tid : INF, sh.tmp32);
+                if (first == INF) break;
+                rdir = sh.dir[first];
+                const bool stops = tid > (int)first && tid < (int)wn &&
+                                   ((dir >= DIR_ALLOC && dir != rdir) || prev_same >= (int)cur);
+                end = block_min(stops ? (uint32_t)tid : wn, sh.tmp32);
+            }
             const bool in_run = tid >= (int)cur && tid < (int)end && dir == rdir;
             unsigned long long tot;
 
@@ -294,14 +439,12 @@ __device__ void step_body(const Geom &g, Shared<NT> &sh, const avmp_op *__restri
                         st = AVMP_ST_OK;
                     } else st = AVMP_ST_BAD_REQ;
                 }
-                const unsigned long long incl =
-                    block_incl_scan(((unsigned long long)nsu << 32) | nk, sh.tmp64, &tot);
+                const unsigned long long incl = scan1<NT>(((unsigned long long)nsu << 32) | nk, sh.scan_part, flip_s, &tot);
                 sh.excl_k[tid] = (uint32_t)incl - nk;
                 sh.excl_s[tid] = (uint32_t)(incl >> 32) - nsu;
                 if (tid == NT - 1) { sh.excl_k[NT] = (uint32_t)tot; sh.excl_s[NT] = (uint32_t)(tot >> 32); }
                 __syncthreads();
                 const uint32_t Tk = (uint32_t)tot, Ts = (uint32_t)(tot >> 32);
-                const uint32_t fk = sc.nfree[0], vk = sc.nvfree[0], fs = sc.nfree[1], vs = sc.nvfree[1];
                 for (uint32_t u = tid; u < Tk; u += NT) {
                     const uint32_t idx = find_owner(sh.excl_k, cur, end, 0u, u);
                     const uint32_t j = u - sh.excl_k[idx];
@@ -309,8 +452,8 @@ __device__ void step_body(const Geom &g, Shared<NT> &sh, const avmp_op *__restri
                     const uint32_t slot = g.VT[0][vid];
                     g.VT[0][vid] = INF;
                     g.OW[0][slot] = INF;
-                    g.S[0][fk + u] = slot;
-                    g.W[0][vk + u] = vid;
+                    g.S[0][nf0 + u] = slot;
+                    g.W[0][nv0 + u] = vid;
                 }
                 for (uint32_t u = tid; u < Ts; u += NT) {
                     const uint32_t idx = find_owner(sh.excl_s, cur, end, 0u, u);
@@ -319,19 +462,15 @@ __device__ void step_body(const Geom &g, Shared<NT> &sh, const avmp_op *__restri
                     const uint32_t slot = g.VT[1][vid];
                     g.VT[1][vid] = INF;
                     g.OW[1][slot] = INF;
-                    g.S[1][fs + u] = slot;
-                    g.W[1][vs + u] = vid;
+                    g.S[1][nf1 + u] = slot;
+                    g.W[1][nv1 + u] = vid;
                 }
                 if (valid) {
                     if (!keep) { g.r_npages[req] = 0; g.r_len[req] = 0; }
                     g.r_state[req] = keep ? AVMP_REQ_KV_ONLY : AVMP_REQ_EMPTY;
                 }
-                __syncthreads();
-                if (tid == 0) {
-                    sc.nfree[0] += Tk; sc.nvfree[0] += Tk;
-                    sc.nfree[1] += Ts; sc.nvfree[1] += Ts;
-                }
-                __syncthreads();
+                nf0 += Tk; nv0 += Tk; nf1 += Ts; nv1 += Ts;
+                __syncthreads();            // the lists and records are in place for what follows
             } else {
                 // ---- alloc run (a4, a5-a9 on shortage) ----
                 uint32_t nk = 0, nsu = 0, new_len = 0;
@@ -359,89 +498,111 @@ __device__ void step_body(const Geom &g, Shared<NT> &sh, const avmp_op *__restri
                         }
                     }
                 }
-                const unsigned long long incl =
-                    block_incl_scan(((unsigned long long)nsu << 32) | nk, sh.tmp64, &tot);
+                const unsigned long long incl = scan1<NT>(((unsigned long long)nsu << 32) | nk, sh.scan_part, flip_s, &tot);
                 sh.excl_k[tid] = (uint32_t)incl - nk;
                 sh.excl_s[tid] = (uint32_t)(incl >> 32) - nsu;
                 if (tid == NT - 1) { sh.excl_k[NT] = (uint32_t)tot; sh.excl_s[NT] = (uint32_t)(tot >> 32); }
                 __syncthreads();
 
-                uint32_t c2 = cur;
-                while (c2 < end) {
-                    // first op of [c2, end) that does not fit, given that all before it do
-                    const uint32_t bk = sh.excl_k[c2], bs = sh.excl_s[c2];
-                    const bool fails = valid && tid >= (int)c2 && tid < (int)end &&
-                                       ((uint32_t)incl - bk > sc.nfree[0] || (uint32_t)(incl >> 32) - bs > sc.nfree[1]);
-                    const uint32_t f = block_min(fails ? (uint32_t)tid : end, sh.tmp32);
-                    if (f > c2) commit_allocs(g, sh, c2, f);
-                    if (valid && tid >= (int)c2 && tid < (int)f) {
+                // demand of the run's ops alone (the scan covers the whole block; ops outside the run add nothing)
+                if ((uint32_t)tot <= nf0 && (uint32_t)(tot >> 32) <= nf1) {
+                    // everything fits: one pass
+                    uint32_t Tk, Ts;
+                    pop_units<NT>(g, sh, cur, end, nf0, nv0, nf1, nv1, Tk, Ts);
+                    if (valid) {
                         g.r_npages[req] = sh.base[tid] + nk;
                         g.r_len[req] = new_len;
                         g.r_state[req] = AVMP_REQ_LIVE;
                         st = AVMP_ST_OK;
                     }
-                    if (f >= end) break;
-
-                    // ---- op f raises CapacityError ----
-                    const uint32_t need_k = sh.excl_k[f + 1] - sh.excl_k[f];
-                    const uint32_t need_s = sh.excl_s[f + 1] - sh.excl_s[f];
-                    const unsigned long long counter = sc.counter_base + (w0 - start) + f + 1ull;
-                    const bool wantA = need_s > sc.nfree[1];
-                    const bool trigA = wantA && would_migrate(g, sc, AVMP_POOL_SSM, counter);
-                    const bool trigB = !trigA && need_k > sc.nfree[0] && would_migrate(g, sc, AVMP_POOL_KV, counter);
-                    if ((trigA || trigB) && sc.migs_done >= 1u) {
-                        // a second migration must wait for the first one's copies: stop here
-                        __syncthreads();
-                        if (tid == 0) { sc.abort = 1; sc.abort_idx = f; }
-                        __syncthreads();
-                        break;
-                    }
-                    const uint32_t migs_before = sc.migs_done;
-                    if (tid == 0) sc.t_fail = clock64();
-                    if (wantA) capacity_error(g, sh, AVMP_POOL_SSM, counter);
-                    if (need_k > sc.nfree[0]) capacity_error(g, sh, AVMP_POOL_KV, counter);
-                    const bool fits = need_s <= sc.nfree[1] && need_k <= sc.nfree[0];
-                    if (fits) {
-                        commit_allocs(g, sh, f, f + 1);
-                        if (tid == (int)f) {
+                    nf0 -= Tk; nv0 -= Tk; nf1 -= Ts; nv1 -= Ts;
+                    __syncthreads();        // the tables are in place for what follows
+                } else {
+                    // shortage somewhere in the run: the counts move to shared memory for the handler
+                    if (tid == 0) { sc.nfree[0] = nf0; sc.nvfree[0] = nv0; sc.nfree[1] = nf1; sc.nvfree[1] = nv1; }
+                    __syncthreads();
+                    uint32_t c2 = cur;
+                    while (c2 < end) {
+                        // first op of [c2, end) that does not fit, given that all before it do
+                        const uint32_t bk = sh.excl_k[c2], bs = sh.excl_s[c2];
+                        const bool fails = valid && tid >= (int)c2 && tid < (int)end &&
+                                           ((uint32_t)incl - bk > sc.nfree[0] || (uint32_t)(incl >> 32) - bs > sc.nfree[1]);
+                        const uint32_t f = min1<NT>(fails ? (uint32_t)tid : end, sh.min_part, flip_m);
+                        if (f > c2) commit_allocs(g, sh, c2, f);
+                        if (valid && tid >= (int)c2 && tid < (int)f) {
                             g.r_npages[req] = sh.base[tid] + nk;
                             g.r_len[req] = new_len;
                             g.r_state[req] = AVMP_REQ_LIVE;
                             st = AVMP_ST_OK;
                         }
-                    } else {
-                        if (tid == (int)f) { st = AVMP_ST_OOM; sc.n_oom += 1; }
-                        __syncthreads();
+                        if (f >= end) break;
+
+                        // ---- op f raises CapacityError ----
+                        const uint32_t need_k = sh.excl_k[f + 1] - sh.excl_k[f];
+                        const uint32_t need_s = sh.excl_s[f + 1] - sh.excl_s[f];
+                        const unsigned long long counter = sc.counter_base + (w0 - start) + f + 1ull;
+                        const bool wantA = need_s > sc.nfree[1];
+                        const bool trigA = wantA && would_migrate(g, sc, AVMP_POOL_SSM, counter);
+                        const bool trigB = !trigA && need_k > sc.nfree[0] && would_migrate(g, sc, AVMP_POOL_KV, counter);
+                        if ((trigA || trigB) && sc.migs_done >= 1u) {
+                            // a second migration must wait for the first one's copies: stop here
+                            __syncthreads();
+                            if (tid == 0) { sc.abort = 1; sc.abort_idx = f; }
+                            __syncthreads();
+                            break;
+                        }
+                        const uint32_t migs_before = sc.migs_done;
+                        if (tid == 0) sc.t_fail = clock64();
+                        if (wantA) capacity_error(g, sh, AVMP_POOL_SSM, counter);
+                        if (need_k > sc.nfree[0]) capacity_error(g, sh, AVMP_POOL_KV, counter);
+                        const bool fits = need_s <= sc.nfree[1] && need_k <= sc.nfree[0];
+                        if (fits) {
+                            commit_allocs(g, sh, f, f + 1);
+                            if (tid == (int)f) {
+                                g.r_npages[req] = sh.base[tid] + nk;
+                                g.r_len[req] = new_len;
+                                g.r_state[req] = AVMP_REQ_LIVE;
+                                st = AVMP_ST_OK;
+                            }
+                        } else {
+                            if (tid == (int)f) { st = AVMP_ST_OOM; sc.n_oom += 1; }
+                            __syncthreads();
+                        }
+                        // time decomposition (paper Section 4.3): cycles spent on this failure go to the
+                        // migration bucket if it migrated, to the OOM-retry bucket otherwise
+                        if (tid == 0) {
+                            const unsigned long long dt = (unsigned long long)(clock64() - sc.t_fail);
+                            if (sc.migs_done != migs_before) sc.cyc_mig += dt; else sc.cyc_oom += dt;
+                        }
+                        c2 = f + 1;
                     }
-                    // time decomposition (paper Section 4.3): cycles spent on this failure go to the
-                    // migration bucket if it migrated, to the OOM-retry bucket otherwise
-                    if (tid == 0) {
-                        const unsigned long long dt = (unsigned long long)(clock64() - sc.t_fail);
-                        if (sc.migs_done != migs_before) sc.cyc_mig += dt; else sc.cyc_oom += dt;
-                    }
-                    c2 = f + 1;
+                    __syncthreads();
+                    nf0 = sc.nfree[0]; nv0 = sc.nvfree[0]; nf1 = sc.nfree[1]; nv1 = sc.nvfree[1];
+                    aborted = sc.abort != 0;
+                    if (aborted) break;
                 }
-                if (sc.abort) break;
             }
             cur = end;
         }
         // ---- statuses of this window ----
-        const uint32_t limit = sc.abort ? sc.abort_idx : wn;
+        const uint32_t limit = aborted ? sc.abort_idx : wn;
         const bool decided = tid < (int)limit;
         if (decided) status[w0 + tid] = st;
-        const int n_inv = __syncthreads_count(decided && st >= AVMP_ST_BAD_REQ && st != ST_PENDING);
-        if (tid == 0) sc.n_invalid += n_inv;
-        __syncthreads();
-        if (sc.abort) { done_upto = w0 + sc.abort_idx; break; }
+        const uint32_t n_inv = __popc(__ballot_sync(0xFFFFFFFFu, decided && st >= AVMP_ST_BAD_REQ && st != ST_PENDING));
+        if (lane == 0 && n_inv) atomicAdd(&sh.n_inv, n_inv);
+        if (aborted) { done_upto = w0 + sc.abort_idx; break; }
+        if (w0 + NT < n_ops) __syncthreads();       // the next window reuses dir / req / w_shape
     }
 
+    __syncthreads();                                // n_inv and the handler's scalars are final
     if (tid == 0) {
         ds->last_rebalance_op = sc.last; ds->n_oom = sc.n_oom; ds->n_capacity_error = sc.n_ce;
         ds->n_rebalance = sc.n_reb; ds->migrated_bytes = sc.migrated; ds->wasted_bytes = sc.wasted;
         ds->relocated_blocks = sc.reloc_blocks; ds->relocated_bytes = sc.reloc_bytes;
-        ds->gap_bytes = sc.gap; ds->n_invalid = sc.n_invalid;
+        ds->gap_bytes = sc.gap; ds->n_invalid = sc.n_invalid + sh.n_inv;
         ds->op_counter = sc.counter_base + (done_upto - start);
-        for (int p = 0; p < 2; ++p) { ds->cap[p] = sc.cap[p]; ds->n_free[p] = sc.nfree[p]; ds->n_vfree[p] = sc.nvfree[p]; }
+        ds->cap[0] = sc.cap[0]; ds->cap[1] = sc.cap[1];
+        ds->n_free[0] = nf0; ds->n_free[1] = nf1; ds->n_vfree[0] = nv0; ds->n_vfree[1] = nv1;
         ds->fsm = sc.fsm;
         ds->resume_idx = done_upto;
         ds->cyc_total += (unsigned long long)(clock64() - sc.t_start);

@@ -36,6 +36,20 @@ class GpuEngine:
         self.ctx.step(d_ops, n, d_st)
         return d_st.cpu().numpy().view(np.uint32)
 
+    def step_translate(self, ops: np.ndarray, handles):
+        """avmp_step_translate -> (statuses, pool, offset, error items, arena offset)."""
+        h = np.ascontiguousarray(handles, dtype=np.uint32)
+        n, nh = len(ops), len(h)
+        d_st = torch.full((max(n, 1),), 0xEE, dtype=torch.int32, device=self.dev)
+        pool = torch.zeros(max(nh, 1), dtype=torch.int32, device=self.dev)
+        off = torch.zeros(max(nh, 1), dtype=torch.int64, device=self.dev)
+        aoff = torch.zeros(max(nh, 1), dtype=torch.int64, device=self.dev)
+        before = self.ctx.stats()["error_count"]
+        self.ctx.step_translate(self._dev(ops), n, d_st, self._dev(h), nh, pool, off, aoff)
+        bad = self.ctx.stats()["error_count"] - before
+        return (d_st.cpu().numpy().view(np.uint32)[:n], pool.cpu().numpy().view(np.uint32)[:nh],
+                off.cpu().numpy().view(np.uint64)[:nh], bad, aoff.cpu().numpy().view(np.uint64)[:nh])
+
     def step_host(self, ops: np.ndarray) -> np.ndarray:
         ops = np.ascontiguousarray(ops)
         st = np.full(len(ops), 0xEE, np.uint32)
@@ -97,20 +111,25 @@ class GpuEngine:
         return st.cpu().numpy(), cv.cpu().numpy()
 
     def gather_step(self, kv_first, kv_n, ssm_first, ssm_n, reqs, capacity_tokens):
-        """Both gathers in one launch -> (K [kv_n][cap][row], V, cu_seqlens, state [ssm_n][n][..], conv, error items)."""
+        """Both gathers in one launch -> (K [kv_n][cap][row], V, cu_seqlens, state [ssm_n][n][..], conv, error items).
+        Layer strides are rounded up to the 16 bytes the entry point asks for."""
         r = np.ascontiguousarray(reqs, dtype=np.uint32)
-        row, n, cap = self.model.kv_row_bytes, max(len(r), 1), max(capacity_tokens, 1)
-        out_k = torch.zeros((kv_n, cap, row), dtype=torch.uint8, device=self.dev)
-        out_v = torch.zeros((kv_n, cap, row), dtype=torch.uint8, device=self.dev)
+        m = self.model
+        row, n, cap = m.kv_row_bytes, max(len(r), 1), max(capacity_tokens, 1)
+        up = lambda x: (x + 15) // 16 * 16
+        ks, ss, cs = up(cap * row), up(n * m.state_bytes), up(n * m.conv_bytes)
+        out_k = torch.zeros((kv_n, ks), dtype=torch.uint8, device=self.dev)
+        out_v = torch.zeros((kv_n, ks), dtype=torch.uint8, device=self.dev)
         cu = torch.zeros(len(r) + 1, dtype=torch.int32, device=self.dev)
-        st = torch.zeros((ssm_n, n, self.model.state_bytes), dtype=torch.uint8, device=self.dev)
-        cv = torch.zeros((ssm_n, n, self.model.conv_bytes), dtype=torch.uint8, device=self.dev)
+        st = torch.zeros((ssm_n, ss), dtype=torch.uint8, device=self.dev)
+        cv = torch.zeros((ssm_n, cs), dtype=torch.uint8, device=self.dev)
         before = self.ctx.stats()["error_count"]
-        self.ctx.gather_step(self._dev(r), len(r), kv_first, kv_n, out_k, out_v, cap * row, capacity_tokens, cu,
-                             ssm_first, ssm_n, st, n * self.model.state_bytes, cv, n * self.model.conv_bytes)
+        self.ctx.gather_step(self._dev(r), len(r), kv_first, kv_n, out_k, out_v, ks, capacity_tokens, cu,
+                             ssm_first, ssm_n, st, ss, cv, cs)
         bad = self.ctx.stats()["error_count"] - before
-        return (out_k.cpu().numpy(), out_v.cpu().numpy(), cu.cpu().numpy().view(np.uint32),
-                st.cpu().numpy(), cv.cpu().numpy(), bad)
+        return (out_k.cpu().numpy()[:, :cap * row].reshape(kv_n, cap, row), out_v.cpu().numpy()[:, :cap * row].reshape(kv_n, cap, row),
+                cu.cpu().numpy().view(np.uint32), st.cpu().numpy()[:, :n * m.state_bytes].reshape(ssm_n, n, m.state_bytes),
+                cv.cpu().numpy()[:, :n * m.conv_bytes].reshape(ssm_n, n, m.conv_bytes), bad)
 
     def scatter_kv(self, layer, reqs, tok_start, in_k, in_v) -> int:
         r = np.ascontiguousarray(reqs, dtype=np.uint32)

@@ -1005,3 +1005,49 @@ def test_step_gather_in_one_launch(env, n_list):
         check(1, 2, 7, 3, tot)
         check(3, 1, 11, 1, tot - 1)                               # the last request does not fit: it copies nothing
     g.ctx.clear_error()
+
+
+@pytest.mark.parametrize("name,steps,over", [
+    ("pr1", 500, dict(pool_bytes=24 * W.MiB, concurrency=12, min_rebalance_interval_ops=50, migration_batch_size=6,
+                      n_requests=300)),                                            # relocations in most migrations
+    ("tiny", 60, dict(min_rebalance_interval_ops=1, migration_batch_size=2)),      # several rounds per step
+    ("short_uniform", 300, dict(migration_enabled=False)),                         # no relocation launch at all
+    ("short_uniform", 400, {}),
+])
+def test_step_translate_equals_step_then_translate(env, name, steps, over):
+    """avmp_step_translate (the translation rides on the step's relocation-copy launch): statuses, tables and the
+    translation of a handle list against the tables AFTER the step -- the handles every slot held before the
+    step, so some are dead by then and some were relocated by the step's migration."""
+    w = W.config(name, **over)
+    g, o = _pair(env, w)
+    d = W.ClosedLoopDriver(w)
+    seen = dict(dead=0, handles=0)
+    for _ in range(steps):
+        if d.done:
+            break
+        t = o.tables()
+        held = np.flatnonzero(t["req_state"] != 0)
+        chain = t["req_chain"].reshape(w.max_requests, w.max_pages)
+        ssm = t["req_ssm"].reshape(w.max_requests, -1)
+        handles = np.concatenate([chain[r, :t["req_npages"][r]] for r in held] +
+                                 [ssm[r] for r in held if t["req_state"][r] == 1] + [np.zeros(0, np.uint32)]).astype(np.uint32)
+        ops = d.next_batch()
+        so = o.step(ops)
+        po, oo, bo = o.translate(handles)
+        sg, pg, og, bg, ag = g.step_translate(ops, handles)
+        assert np.array_equal(sg, so) and bg == bo
+        assert np.array_equal(pg, po) and np.array_equal(og, oo)
+        st_ = o.stats()
+        live = po != 0xFFFFFFFF
+        expect = np.where(po == 0, oo, np.uint64(st_["pool_bytes_aligned"] - st_["unit_bytes_ssm"]) - oo)
+        assert np.array_equal(ag[live], expect[live])
+        seen["dead"] += bo
+        seen["handles"] += len(handles)
+        d.feed(so)
+        if d.step % 50 == 0:
+            env["same"](g, o, w, f"step {d.step}")
+        g.ctx.clear_error()
+    env["same"](g, o, w, "end")
+    assert seen["handles"] > 500 and seen["dead"] > 0
+    if w.migration_enabled:
+        assert g.stats()["n_rebalance"] > 0
