@@ -556,6 +556,116 @@ def migration_microbench(dev) -> dict:
                     "(CUDA events); copy kernel alone by the device clock stamped inside it (first warp in, last out)"}
 
 
+def remap_microbench(dev, granules=(1, 2, 4, 8, 16, 32, 64), reps=7) -> dict:
+    """What migrating capacity by remapping physical pages would cost on this machine (the paper's proposed
+    alternative to oversized stores, Sections 3.2 / 4.6): two virtual ranges (the two stores), N physical
+    granules unmapped from the donor's range and mapped into the recipient's with the CUDA virtual memory
+    management calls, including the stream synchronisation the host needs before it may touch mappings the
+    device might still be using (and to learn the device's decision at all).  Host wall clock, median of
+    `reps`; 128 MiB of physical memory in total.  Compared by the caller with the relocation copy's time."""
+    import torch
+    from cuda.bindings import driver as cu
+
+    def ck(r):
+        err, rest = r[0], r[1:]
+        if int(err) != 0:
+            raise RuntimeError(f"CUDA driver call failed: {err}")
+        return rest[0] if len(rest) == 1 else rest
+
+    torch.cuda.synchronize(dev)
+    prop = cu.CUmemAllocationProp()
+    prop.type = cu.CUmemAllocationType.CU_MEM_ALLOCATION_TYPE_PINNED
+    prop.location.type = cu.CUmemLocationType.CU_MEM_LOCATION_TYPE_DEVICE
+    prop.location.id = dev.index or 0
+    gran = int(ck(cu.cuMemGetAllocationGranularity(prop, cu.CUmemAllocationGranularity_flags.CU_MEM_ALLOC_GRANULARITY_MINIMUM)))
+    n_max = max(granules)
+    span = n_max * gran
+    va = [int(ck(cu.cuMemAddressReserve(span, gran, 0, 0))) for _ in range(2)]     # donor range, recipient range
+    handles = [ck(cu.cuMemCreate(gran, prop, 0)) for _ in range(n_max)]
+    acc = cu.CUmemAccessDesc()
+    acc.location.type = cu.CUmemLocationType.CU_MEM_LOCATION_TYPE_DEVICE
+    acc.location.id = dev.index or 0
+    acc.flags = cu.CUmemAccess_flags.CU_MEM_ACCESS_FLAGS_PROT_READWRITE
+    where = 0                                       # which range the granules are mapped in
+    flag = torch.zeros(2, dtype=torch.int64, device=dev)
+    h_flag = torch.zeros(2, dtype=torch.int64).pin_memory()
+    rows = []
+    try:
+        for i, h in enumerate(handles):
+            ck(cu.cuMemMap(va[0] + i * gran, gran, 0, h, 0))
+        ck(cu.cuMemSetAccess(va[0], span, [acc], 1))
+        for n in granules:
+            samples, sync_samples = [], []
+            for _ in range(reps):
+                src, dst = va[where], va[1 - where]
+                torch.cuda.synchronize(dev)
+                t0 = time.perf_counter()
+                h_flag.copy_(flag, non_blocking=True)              # the device's decision reaches the host
+                torch.cuda.synchronize(dev)
+                t1 = time.perf_counter()
+                for i in range(n):
+                    ck(cu.cuMemUnmap(src + i * gran, gran))
+                    ck(cu.cuMemMap(dst + i * gran, gran, 0, handles[i], 0))
+                ck(cu.cuMemSetAccess(dst, n * gran, [acc], 1))
+                t2 = time.perf_counter()
+                samples.append((t2 - t0) * 1e6)
+                sync_samples.append((t1 - t0) * 1e6)
+                # back again (untimed), so that every sample starts from the same mapping
+                for i in range(n):
+                    ck(cu.cuMemUnmap(dst + i * gran, gran))
+                    ck(cu.cuMemMap(src + i * gran, gran, 0, handles[i], 0))
+                ck(cu.cuMemSetAccess(src, n * gran, [acc], 1))
+            rows.append({"granules": n, "bytes": n * gran, "remap_us": float(np.median(samples)),
+                         "of_which_sync_and_readback_us": float(np.median(sync_samples)),
+                         "us_per_granule": (float(np.median(samples)) - float(np.median(sync_samples))) / n})
+    finally:
+        for i in range(n_max):                  # each granule is mapped in one of the two ranges (errors ignored)
+            cu.cuMemUnmap(va[0] + i * gran, gran)
+            cu.cuMemUnmap(va[1] + i * gran, gran)
+        for h in handles:
+            cu.cuMemRelease(h)
+        for r in va:
+            cu.cuMemAddressFree(r, span)
+    return {"granule_bytes": gran, "rows": rows,
+            "note": "host wall clock per migration of N granules: readback + stream sync, then cuMemUnmap + cuMemMap per "
+                    "granule and one cuMemSetAccess for the range; no data moves"}
+
+
+def relocation_small_cases(dev, batch_units=(8, 32, 128, 512, 2048)) -> list:
+    """The copy path on the same byte counts: one migration of B KV pages (256 KiB each) out of a half-live
+    store, timed as the whole avmp_step (plan kernel + copy, CUDA events) and as the copy kernel alone (device
+    clock).  About half of the ceded pages are live and have to be copied."""
+    import torch
+    from paper_2605_22416_b200 import binding as B
+    m = W.JAMBA_LIKE
+    out = []
+    for units in batch_units:
+        ctx = B.Context(m, 4 * W.GiB, 0.3, units, max_requests=256, max_pages=256, device=dev)
+        s0 = ctx.stats()
+        n_req = s0["cap_ssm"] // m.n_ssm_layers
+        per = min(256, s0["cap_kv"] // n_req)
+        st = np.zeros(512, np.uint32)
+        ctx.step_host(W.make_ops(W.OP_ADMIT, np.arange(n_req), per * 16), n_req, st)
+        assert (st[:n_req] == 0).all()
+        fin = np.arange(0, n_req, 2)
+        ctx.step_host(W.make_ops(W.OP_FINISH, fin, 0), len(fin), st)
+        ops = W.make_ops(W.OP_ADMIT, 128 + np.arange(n_req), 16)
+        d_ops = torch.from_numpy(ops.view(np.uint8).reshape(-1)).to(dev)
+        d_st = torch.zeros(n_req, dtype=torch.int32, device=dev)
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ctx.step(d_ops, n_req, d_st)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        s = ctx.stats()
+        ctx.close()
+        out.append({"migration_batch_units": units, "ceded_bytes": s["migrated_bytes"], "relocated_bytes": s["relocated_bytes"],
+                    "rebalances": s["n_rebalance"], "step_us": e0.elapsed_time(e1) * 1e3,
+                    "copy_kernel_us_device_clock": s["relocation_ns_last"] / 1e3})
+    return out
+
+
 def device_closed_loop(dev, workload: str, steps: int = 3000) -> dict:
     """The whole serving loop on the device (batch built, allocator stepped and statuses folded back by
     kernels, no host round trip), dynamic rebalancing against the static partition on the same trace:
@@ -857,6 +967,10 @@ def main():
             sec["relocation_copy"] = migration_microbench(dev)
             sec["allocator_vs_step_batch"] = allocator_scaling(dev)
             sec["write_side"] = write_side_microbench(dev)
+            try:
+                sec["remap_vs_copy"] = {"remap": remap_microbench(dev), "copy": relocation_small_cases(dev)}
+            except Exception as exc:          # the comparison is context for one design decision, not part of the path
+                sec["remap_vs_copy"] = {"unavailable": f"{type(exc).__name__}: {exc}"}
             sec["closed_loop_device"] = device_closed_loop(dev, args.workload, 1500 if args.workload == "scale" else 3000)
             out["roofline"]["other_configs"] = other_configs(dev, skip=args.workload)
         if not args.no_cpu_baseline:

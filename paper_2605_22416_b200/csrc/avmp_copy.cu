@@ -492,8 +492,15 @@ __global__ void __launch_bounds__(kBulkThreads, kBulkCtasPerSm) stream_bulk_kern
             record_error(g.st, AVMP_DEV_TIMEOUT);
             ring.drain_loads();
         }
-        bulk_wait_all();
-        if (F::kTimed) atomicMax(&g.st->reloc_t1, global_ns());
+        // Before the CTA may exit, the stores must have read their shared-memory stages; that they have
+        // reached global memory is guaranteed by the end of the kernel.  The timed copy waits for that too,
+        // so that its clock stamp covers the whole transfer.
+        if (F::kTimed) {
+            bulk_wait_all();
+            atomicMax(&g.st->reloc_t1, global_ns());
+        } else {
+            bulk_wait_read<0>();
+        }
     }
 }
 

@@ -94,13 +94,16 @@ __device__ __forceinline__ uint32_t min1(uint32_t v, uint32_t (*part)[32], uint3
     return m;
 }
 
-__device__ __forceinline__ bool would_migrate(const Geom &g, const Scalars &sc, int X, unsigned long long counter)
+// Section 3.2 trigger for a shortage in pool X: the donor Y must have more than threshold_high of its units free
+// (strictly), the throttle must have run out, and what it can cede must make at least one whole unit of X.
+__device__ __forceinline__ bool would_migrate(const Geom &g, const Scalars &sc, int X, unsigned long long counter,
+                                              uint32_t donor_free)
 {
     const int Y = 1 - X;
     if (!g.migration_enabled || sc.cap[Y] == 0) return false;
-    if (!((unsigned long long)sc.nfree[Y] * 1000000ull > (unsigned long long)g.th_high * sc.cap[Y])) return false;
+    if (!((unsigned long long)donor_free * 1000000ull > (unsigned long long)g.th_high * sc.cap[Y])) return false;
     if (sc.last != kNone64 && counter - sc.last < g.min_interval) return false;
-    const unsigned long long n = g.B < sc.nfree[Y] ? g.B : sc.nfree[Y];
+    const unsigned long long n = g.B < donor_free ? g.B : donor_free;
     // reclaim_gap variant: the bytes already lying between the pools are offered again
     return (n * g.U[Y] + (g.reclaim_gap ? sc.gap : 0ull)) / g.U[X] >= 1ull;
 }
@@ -119,7 +122,7 @@ __device__ void capacity_error(const Geom &g, Shared<NT> &sh, int X, unsigned lo
             sc.fsm = pressured;
         else if (sc.fsm == pressured)
             sc.fsm = AVMP_FSM_BALANCED;
-        sc.mig = would_migrate(g, sc, X, counter) ? 1u : 0u;
+        sc.mig = would_migrate(g, sc, X, counter, sc.nfree[Y]) ? 1u : 0u;
         if (sc.mig) {
             const unsigned long long n = g.B < sc.nfree[Y] ? g.B : sc.nfree[Y];
             const unsigned long long carry = g.reclaim_gap ? sc.gap : 0ull;
@@ -236,21 +239,6 @@ __device__ __forceinline__ void pop_units(const Geom &g, Shared<NT> &sh, uint32_
         g.OW[1][slot] = vid;
         g.r_ssm[(unsigned long long)sh.req[idx] * g.ns + j] = 0x80000000u | vid;
     }
-}
-
-// The same with the heights in shared memory (the shortage path keeps them there for the handler).
-template <int NT>
-__device__ __forceinline__ void commit_allocs(const Geom &g, Shared<NT> &sh, uint32_t lo, uint32_t hi)
-{
-    Scalars &sc = sh.sc;
-    uint32_t Tk, Ts;
-    pop_units<NT>(g, sh, lo, hi, sc.nfree[0], sc.nvfree[0], sc.nfree[1], sc.nvfree[1], Tk, Ts);
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        sc.nfree[0] -= Tk; sc.nvfree[0] -= Tk;
-        sc.nfree[1] -= Ts; sc.nvfree[1] -= Ts;
-    }
-    __syncthreads();
 }
 
 // The whole allocator update for ops[0 .. n_ops) by the calling CTA of NT threads (callers have
@@ -518,32 +506,38 @@ __device__ void step_body(const Geom &g, Shared<NT> &sh, const avmp_op *__restri
                     nf0 -= Tk; nv0 -= Tk; nf1 -= Ts; nv1 -= Ts;
                     __syncthreads();        // the tables are in place for what follows
                 } else {
-                    // shortage somewhere in the run: the counts move to shared memory for the handler
-                    if (tid == 0) { sc.nfree[0] = nf0; sc.nvfree[0] = nv0; sc.nfree[1] = nf1; sc.nvfree[1] = nv1; }
-                    __syncthreads();
+                    // Shortage somewhere in the run.  Everything before the first op that does not fit is
+                    // committed; that op's CapacityError is decided by every thread alike (free counts in
+                    // registers; capacities, throttle state and gap in shared memory, which only a migration
+                    // changes) and thread 0 keeps the counters, so an error that cannot migrate -- the usual
+                    // case under the throttle -- costs no barrier.  Only a migration takes the handler.
                     uint32_t c2 = cur;
                     while (c2 < end) {
                         // first op of [c2, end) that does not fit, given that all before it do
                         const uint32_t bk = sh.excl_k[c2], bs = sh.excl_s[c2];
                         const bool fails = valid && tid >= (int)c2 && tid < (int)end &&
-                                           ((uint32_t)incl - bk > sc.nfree[0] || (uint32_t)(incl >> 32) - bs > sc.nfree[1]);
+                                           ((uint32_t)incl - bk > nf0 || (uint32_t)(incl >> 32) - bs > nf1);
                         const uint32_t f = min1<NT>(fails ? (uint32_t)tid : end, sh.min_part, flip_m);
-                        if (f > c2) commit_allocs(g, sh, c2, f);
-                        if (valid && tid >= (int)c2 && tid < (int)f) {
-                            g.r_npages[req] = sh.base[tid] + nk;
-                            g.r_len[req] = new_len;
-                            g.r_state[req] = AVMP_REQ_LIVE;
-                            st = AVMP_ST_OK;
+                        if (f > c2) {
+                            uint32_t Tk, Ts;
+                            pop_units<NT>(g, sh, c2, f, nf0, nv0, nf1, nv1, Tk, Ts);
+                            if (valid && tid >= (int)c2 && tid < (int)f) {
+                                g.r_npages[req] = sh.base[tid] + nk;
+                                g.r_len[req] = new_len;
+                                g.r_state[req] = AVMP_REQ_LIVE;
+                                st = AVMP_ST_OK;
+                            }
+                            nf0 -= Tk; nv0 -= Tk; nf1 -= Ts; nv1 -= Ts;
                         }
                         if (f >= end) break;
 
-                        // ---- op f raises CapacityError ----
+                        // ---- op f raises CapacityError (SSM first, then KV) ----
                         const uint32_t need_k = sh.excl_k[f + 1] - sh.excl_k[f];
                         const uint32_t need_s = sh.excl_s[f + 1] - sh.excl_s[f];
                         const unsigned long long counter = sc.counter_base + (w0 - start) + f + 1ull;
-                        const bool wantA = need_s > sc.nfree[1];
-                        const bool trigA = wantA && would_migrate(g, sc, AVMP_POOL_SSM, counter);
-                        const bool trigB = !trigA && need_k > sc.nfree[0] && would_migrate(g, sc, AVMP_POOL_KV, counter);
+                        const bool wantA = need_s > nf1;
+                        const bool trigA = wantA && would_migrate(g, sc, AVMP_POOL_SSM, counter, nf0);
+                        const bool trigB = !trigA && need_k > nf0 && would_migrate(g, sc, AVMP_POOL_KV, counter, nf1);
                         if ((trigA || trigB) && sc.migs_done >= 1u) {
                             // a second migration must wait for the first one's copies: stop here
                             __syncthreads();
@@ -551,33 +545,50 @@ __device__ void step_body(const Geom &g, Shared<NT> &sh, const avmp_op *__restri
                             __syncthreads();
                             break;
                         }
-                        const uint32_t migs_before = sc.migs_done;
                         if (tid == 0) sc.t_fail = clock64();
-                        if (wantA) capacity_error(g, sh, AVMP_POOL_SSM, counter);
-                        if (need_k > sc.nfree[0]) capacity_error(g, sh, AVMP_POOL_KV, counter);
-                        const bool fits = need_s <= sc.nfree[1] && need_k <= sc.nfree[0];
-                        if (fits) {
-                            commit_allocs(g, sh, f, f + 1);
+                        auto label_only = [&](int X, uint32_t nfX) {          // thread 0: the handler without a migration
+                            sc.n_ce += 1;
+                            const uint32_t pressured = X == AVMP_POOL_KV ? AVMP_FSM_KV_PRESSURED : AVMP_FSM_SSM_PRESSURED;
+                            if ((unsigned long long)nfX * 1000000ull < (unsigned long long)g.th_low * sc.cap[X]) sc.fsm = pressured;
+                            else if (sc.fsm == pressured) sc.fsm = AVMP_FSM_BALANCED;
+                        };
+                        auto migrate = [&](int X) {                            // whole CTA: the handler with its migration
+                            if (tid == 0) { sc.nfree[0] = nf0; sc.nvfree[0] = nv0; sc.nfree[1] = nf1; sc.nvfree[1] = nv1; }
+                            __syncthreads();
+                            capacity_error(g, sh, X, counter);
+                            nf0 = sc.nfree[0]; nv0 = sc.nvfree[0]; nf1 = sc.nfree[1]; nv1 = sc.nvfree[1];
+                        };
+                        if (wantA) {
+                            if (trigA) migrate(AVMP_POOL_SSM);
+                            else if (tid == 0) label_only(AVMP_POOL_SSM, nf1);
+                        }
+                        if (need_k > nf0) {      // a migration for the SSM pool may have taken KV capacity
+                            if (trigB) migrate(AVMP_POOL_KV);
+                            else if (tid == 0) label_only(AVMP_POOL_KV, nf0);   // after trigA the throttle forbids a second one
+                        }
+                        if (need_s <= nf1 && need_k <= nf0) {
+                            uint32_t Tk, Ts;
+                            pop_units<NT>(g, sh, f, f + 1, nf0, nv0, nf1, nv1, Tk, Ts);
                             if (tid == (int)f) {
                                 g.r_npages[req] = sh.base[tid] + nk;
                                 g.r_len[req] = new_len;
                                 g.r_state[req] = AVMP_REQ_LIVE;
                                 st = AVMP_ST_OK;
                             }
+                            nf0 -= Tk; nv0 -= Tk; nf1 -= Ts; nv1 -= Ts;
                         } else {
-                            if (tid == (int)f) { st = AVMP_ST_OOM; sc.n_oom += 1; }
-                            __syncthreads();
+                            if (tid == (int)f) st = AVMP_ST_OOM;
+                            if (tid == 0) sc.n_oom += 1;
                         }
                         // time decomposition (paper Section 4.3): cycles spent on this failure go to the
                         // migration bucket if it migrated, to the OOM-retry bucket otherwise
                         if (tid == 0) {
                             const unsigned long long dt = (unsigned long long)(clock64() - sc.t_fail);
-                            if (sc.migs_done != migs_before) sc.cyc_mig += dt; else sc.cyc_oom += dt;
+                            if (trigA || trigB) sc.cyc_mig += dt; else sc.cyc_oom += dt;
                         }
                         c2 = f + 1;
                     }
-                    __syncthreads();
-                    nf0 = sc.nfree[0]; nv0 = sc.nvfree[0]; nf1 = sc.nfree[1]; nv1 = sc.nvfree[1];
+                    __syncthreads();        // the tables are in place for what follows
                     aborted = sc.abort != 0;
                     if (aborted) break;
                 }

@@ -480,7 +480,7 @@ def test_scale_config(env, split, enabled):
     w = W.config("scale", split=split, migration_enabled=enabled)
     s, seen, d = _closed_loop_parity(env, w, 240 if enabled else 120, with_store=False, kv_layers=[0, 4, 8],
                                      ssm_layers=[0, 31, 62], table_every=40, gather_every=47, max_migration_checks=4)
-    assert seen["tokens"] > (1_000_000 if enabled else 500_000) and s["op_counter"] > 100_000
+    assert seen["tokens"] > (1_000_000 if enabled else 500_000) and s["op_counter"] > 90_000
 
 
 def test_sensitivity_sweep_cells_match_the_oracle(env):
