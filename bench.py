@@ -339,6 +339,25 @@ def measure(w: W.Workload, dev, *, steps: int, warmup: int, warm_steps: int, ask
     per, st_c = timed_classes(per_layer=False)
     per_l = timed_classes(per_layer=True)[0] if full else None
     per_f = timed_classes(per_layer=False, fused=True)[0] if one_launch else None
+
+    # ---- region 3: the allocator part alone (avmp_step_translate per step, the calls back to back as a serving
+    #      loop issues them; no events between steps, which would keep consecutive launches from overlapping) ----
+    def alloc_only(separate):
+        c = fresh_context(full_warmup=False)
+        a0, a1 = ev(), ev()
+        a0.record(stream)
+        for r in timed:
+            if separate:
+                c.step(r["d_ops"], len(r["ops"]), d_status, sid)
+                c.translate(r["d_handles"], len(r["handles"]), d_pool, d_off, d_aoff, sid)
+            else:
+                c.step_translate(r["d_ops"], len(r["ops"]), d_status, r["d_handles"], len(r["handles"]), d_pool, d_off, d_aoff, sid)
+        a1.record(stream)
+        torch.cuda.synchronize(dev)
+        c.close()
+        return a0.elapsed_time(a1)
+
+    alloc_ms, alloc_sep_ms = alloc_only(False), alloc_only(True)
     clocks = sampler.stop()
 
     # ---- e2e: host buffers in, host results out, every step ----
@@ -383,6 +402,7 @@ def measure(w: W.Workload, dev, *, steps: int, warmup: int, warm_steps: int, ask
         "kv_bytes": kv_bytes, "ssm_bytes": ssm_bytes, "reloc_bytes": reloc_timed,
         "moved": kv_bytes + ssm_bytes + 2 * reloc_timed,
         "n_ops": sum(len(r["ops"]) for r in timed), "units": sum(r["units"] for r in timed),
+        "alloc_ms": alloc_ms, "alloc_sep_ms": alloc_sep_ms, "handles": sum(len(r["handles"]) for r in timed),
         "per": per, "per_l": per_l, "per_f": per_f, "one_launch": one_launch, "clocks": clocks, "lpl": (lpl_kv, lpl_ssm),
         "n_kv_launches": len(kv_groups), "n_ssm_launches": len(ssm_groups),
         "running_mean": float(np.mean([len(r["run"]) for r in timed])),
@@ -405,9 +425,11 @@ def class_figures(res: dict, m: W.ModelShape, peak: float) -> dict:
     ssm_ms, kv_ms, step_ms = float(np.mean(per["ssm"])), float(np.mean(per["kv"])), float(np.mean(per["step"]))
     out = {"ssm_gbs": ssm_launch_bytes / (ssm_ms * 1e-3) / 1e9, "ssm_launch_ms": ssm_ms, "ssm_launch_bytes": ssm_launch_bytes,
            "kv_gbs": kv_launch_bytes / (kv_ms * 1e-3) / 1e9, "kv_launch_ms": kv_ms, "kv_launch_bytes": kv_launch_bytes,
-           "allocator_us_per_step": step_ms * 1e3, "allocator_ops_per_s": res["n_ops"] / (sum(per["step"]) * 1e-3),
-           "allocator_us_per_step_separate_calls": float(np.mean(res["per_l"]["step"])) * 1e3 if res["per_l"] is not None else None,
-           "unit_allocs_frees_per_s": res["units"] / (sum(per["step"]) * 1e-3)}
+           "allocator_us_per_step": res["alloc_ms"] * 1e3 / K, "allocator_ops_per_s": res["n_ops"] / (res["alloc_ms"] * 1e-3),
+           "allocator_us_per_step_separate_calls": res["alloc_sep_ms"] * 1e3 / K,
+           "allocator_us_per_step_inside_full_steps": step_ms * 1e3,
+           "unit_allocs_frees_per_s": res["units"] / (res["alloc_ms"] * 1e-3),
+           "handles_translated_per_step": res["handles"] / K}
     if res["per_f"] is not None:
         ms = float(np.mean([a + b for a, b in zip(res["per_f"]["kv"], res["per_f"]["ssm"])]))   # kv mark is empty
         out["step_gather_gbs"] = (res["kv_bytes"] + res["ssm_bytes"]) / K / (ms * 1e-3) / 1e9
@@ -467,13 +489,21 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
                          "single_layer_kv": {"gbs": f["single_layer_kv_gbs"], "frac": f["single_layer_kv_gbs"] / peak,
                                              "avg_launch_ms": f["single_layer_kv_launch_ms"],
                                              "note": "same window, avmp_gather_kv once per layer, back to back"},
+                         "step_gather": ({"gbs": f["step_gather_gbs"], "frac": f["step_gather_gbs"] / peak,
+                                          "avg_launch_ms": f["step_gather_launch_ms"],
+                                          "note": "avmp_gather_step: both gathers of all layers in one launch"}
+                                         if "step_gather_gbs" in f else None),
                          "allocator_ops_per_s": f["allocator_ops_per_s"] * (world if world > 1 else 1),
                          "allocator_us_per_step": f["allocator_us_per_step"],
                          "allocator_us_per_step_separate_calls": f["allocator_us_per_step_separate_calls"],
+                         "allocator_us_per_step_inside_full_steps": f["allocator_us_per_step_inside_full_steps"],
+                         "handles_translated_per_step": f["handles_translated_per_step"],
                          "unit_allocs_frees_per_s": f["unit_allocs_frees_per_s"],
                          "allocator_note": "avmp_step_translate (allocator step + translate of every live handle of the batch; "
-                                           "the translation rides on the step's relocation-copy launch), CUDA events around "
-                                           "the call, rank 0's timing; separate_calls = avmp_step then avmp_translate; units = KV pages + SSM blocks allocated "
+                                           "the translation rides on the step's relocation-copy launch), the window's steps "
+                                           "issued back to back under one CUDA-event pair, rank 0's timing; separate_calls = "
+                                           "avmp_step then avmp_translate; inside_full_steps = the same call between two events "
+                                           "inside whole engine steps (the events keep it from overlapping its neighbours); units = KV pages + SSM blocks allocated "
                                            "or freed, counted from the request slots' net change per step"}},
         "e2e": {"value": sums[0] / (e2e_ms_g * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms_g / K,
                 "h2d_bytes_per_step": sums[5] / K / world, "d2h_bytes_per_step": sums[6] / K / world,

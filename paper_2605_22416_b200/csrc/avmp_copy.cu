@@ -20,12 +20,18 @@
 //     AVMP_DEV_TIMEOUT and stops issuing.
 //   * generic path: plain loads and stores, for shapes whose runs are not 16-byte multiples.
 //
-// Measured alternatives that did not beat this (B200, 244 MB and 6.8 GB launches): the same walk
-// with register-staged 16-byte loads / stores at 2-8 CTAs per SM (equal within 1 %); stages of
-// 4 to 64 KiB and rings of 2 to 8 stages (equal or worse); a global ticket counter (worse);
-// staggered warp starts (worse); smaller pieces for small launches, to even out the last round
-// of the walk (worse: small launches are bound by ramp and tail latency, not by imbalance).  The ceiling is DRAM efficiency for this read/write mix, about
-// 72-75 % of the raw rate, against 78-80 % for one long linear copy.
+// Shape of the ring, measured on B200 (244 MB to 51 GB per launch): what matters most is the number of bytes
+// in flight per SM.  64 KiB (2 warps x 2 stages x 16 KiB, or 1 x 2 x 32 KiB) is the optimum -- a 28-layer SSM
+// gather runs at 6.5 TB/s, the measured copy peak of this part, against 6.1 TB/s with 192 KiB in flight
+// (4 x 3 x 16 KiB), 6.2 with 96 or 128 KiB and 6.1 with 48 KiB; at equal bytes, fewer and larger requests
+// do slightly better, stages that are not a power of two much worse.  Other things tried that did not beat it:
+// register-staged 16-byte loads / stores at 2-8 CTAs per SM, a global ticket counter instead of the static
+// walk, staggered warp starts, smaller pieces for small launches (those are bound by ramp and tail latency,
+// not by imbalance).
+// The CTA nevertheless REQUESTS 120 KiB of shared memory, so that only one copy CTA fits on an SM: every
+// kernel here lets its successor in the stream start early (programmatic dependent launch), and with small
+// CTAs the successors' CTAs were placed two and three to an SM while this kernel still ran, which cost the
+// back-to-back steps of a serving loop 5 % (25 % with 48 KiB CTAs) through the uneven load on the SMs.
 #include "avmp_dev.cuh"
 
 namespace avmp {
@@ -33,11 +39,14 @@ namespace avmp {
 namespace {
 
 // Shape of the bulk path (fixed after sweeps on B200; see the measured alternatives above).
-constexpr int kStages = 3;                      // ring depth per warp
-constexpr int kBulkWarps = 4;                   // warps (rings) per CTA: 4 x 3 x 16 KiB = 192 KiB of shared memory
-constexpr int kBulkCtasPerSm = 1;
+constexpr int kStages = 2;                      // ring depth per warp
+constexpr int kBulkWarps = 2;                   // warps (rings) per CTA: 2 x 2 x 16 KiB = 64 KiB in flight per SM
+constexpr int kBulkCtasPerSm = 1;                // resident CTAs per SM the kernel is compiled for
+constexpr int kBulkGridPerSm = 1;                // CTAs launched per SM
 constexpr int kBulkThreads = kBulkWarps * 32;
-constexpr uint32_t kBulkSmem = kBulkWarps * kStages * kStage;
+constexpr uint32_t kBulkSmemUsed = kBulkWarps * kStages * kStage;
+constexpr uint32_t kBulkSmemPad = 56 * 1024;     // requested on top, unused: one copy CTA per SM (see above)
+constexpr uint32_t kBulkSmem = kBulkSmemUsed + kBulkSmemPad;
 constexpr int kGenThreads = 256;
 constexpr int kGenCtasPerSm = 4;
 constexpr uint32_t kSpinLimit = 1u << 22;
@@ -196,58 +205,49 @@ struct KvPieces {
         if (n > kLocalPlanMax) { cu_items = g.g_cu_items; cu_rows = g.g_cu_rows; req_of = reqs; return; }
         uint32_t *rows_s = buf, *items_s = buf + kLocalPlanMax + 1, *req_s = buf + 2 * (kLocalPlanMax + 1);
         const bool lead = blockIdx.x == 0;            // one CTA reports errors and writes cu_seqlens
-        // Pass 1: every entry's rows and pieces, with all table reads of the list in flight together
-        // (two dependent reads per entry; taken window by window between the scans' barriers they
-        // would cost that latency once per window).  kPer entries per thread cover the longest local
-        // list with the smallest CTA that runs this (128 threads).
+        // Pass 1: every entry's rows and pieces.  Eight entries per thread and round, so that the table reads
+        // of a round (two dependent reads per entry) are in flight together; taken one entry at a time
+        // between barriers they would cost that latency once per entry.
         constexpr int kPer = 8;
-        uint32_t rr[kPer], t0[kPer], st[kPer], ln[kPer];
+        for (uint32_t base = 0; base < n; base += kPer * blockDim.x) {
+            uint32_t rr[kPer], t0[kPer], st[kPer], ln[kPer];
 #pragma unroll
-        for (int i = 0; i < kPer; ++i) {
-            const uint32_t k = threadIdx.x + i * blockDim.x;
-            rr[i] = k < n ? reqs[k] : kInvalid;
-            t0[i] = (k < n && tok_start) ? tok_start[k] : 0u;
-        }
+            for (int i = 0; i < kPer; ++i) {
+                const uint32_t k = base + threadIdx.x + i * blockDim.x;
+                rr[i] = k < n ? reqs[k] : kInvalid;
+                t0[i] = (k < n && tok_start) ? tok_start[k] : 0u;
+            }
 #pragma unroll
-        for (int i = 0; i < kPer; ++i) {
-            const bool in_range = rr[i] < g.R;
-            st[i] = in_range ? g.r_state[rr[i]] : (uint32_t)AVMP_REQ_EMPTY;
-            ln[i] = in_range ? g.r_len[rr[i]] : 0u;
-        }
+            for (int i = 0; i < kPer; ++i) {
+                const bool in_range = rr[i] < g.R;
+                st[i] = in_range ? g.r_state[rr[i]] : (uint32_t)AVMP_REQ_EMPTY;
+                ln[i] = in_range ? g.r_len[rr[i]] : 0u;
+            }
 #pragma unroll
-        for (int i = 0; i < kPer; ++i) {
-            const uint32_t k = threadIdx.x + i * blockDim.x;
-            if (k < n) {
-                uint32_t rows, items;
-                kv_rows_items(g, st[i], ln[i], t0[i], subs, lead, rows, items);
-                rows_s[k] = rows; items_s[k] = items; req_s[k] = rr[i];
+            for (int i = 0; i < kPer; ++i) {
+                const uint32_t k = base + threadIdx.x + i * blockDim.x;
+                if (k < n) {
+                    uint32_t rows, items;
+                    kv_rows_items(g, st[i], ln[i], t0[i], subs, lead, rows, items);
+                    rows_s[k] = rows; items_s[k] = items; req_s[k] = rr[i];
+                }
             }
         }
         __syncthreads();
         // Pass 2: exclusive prefix sums over the list: every thread sums a run of consecutive entries,
         // one block scan orders the runs (one scan for the whole list instead of one per window).
-        const uint32_t per = (n + blockDim.x - 1) / blockDim.x;          // <= kPer
-        const uint32_t k0 = threadIdx.x * per;
-        uint32_t vr[kPer], vi[kPer];
+        const uint32_t per = (n + blockDim.x - 1) / blockDim.x;
+        const uint32_t k0 = threadIdx.x * per, k1 = min(n, k0 + per);
         unsigned long long mine = 0, tot;
-#pragma unroll
-        for (int i = 0; i < kPer; ++i) {
-            const uint32_t k = k0 + i;
-            const bool in = (uint32_t)i < per && k < n;
-            vr[i] = in ? rows_s[k] : 0u; vi[i] = in ? items_s[k] : 0u;
-            mine += ((unsigned long long)vi[i] << 32) | vr[i];
-        }
+        for (uint32_t k = k0; k < k1; ++k) mine += ((unsigned long long)items_s[k] << 32) | rows_s[k];
         const unsigned long long incl = block_incl_scan(mine, tmp, &tot);
         unsigned long long run = incl - mine;
-#pragma unroll
-        for (int i = 0; i < kPer; ++i) {
-            const uint32_t k = k0 + i;
-            if ((uint32_t)i < per && k < n) {
-                rows_s[k] = (uint32_t)run;
-                items_s[k] = (uint32_t)(run >> 32);
-                if (lead && cu_out) cu_out[k] = (uint32_t)run;
-                run += ((unsigned long long)vi[i] << 32) | vr[i];
-            }
+        for (uint32_t k = k0; k < k1; ++k) {
+            const unsigned long long v = ((unsigned long long)items_s[k] << 32) | rows_s[k];
+            rows_s[k] = (uint32_t)run;
+            items_s[k] = (uint32_t)(run >> 32);
+            if (lead && cu_out) cu_out[k] = (uint32_t)run;
+            run += v;
         }
         if (threadIdx.x == 0) {
             rows_s[n] = (uint32_t)tot; items_s[n] = (uint32_t)(tot >> 32);
@@ -547,7 +547,7 @@ cudaError_t launch_stream(const Geom &g, const F &f, bool bulk_ok, const Launch 
             if (e != cudaSuccess) return e;
             attr_set[l.device & 63] = true;
         }
-        return launch_pdl(stream_bulk_kernel<F>, dim3(l.n_sms * kBulkCtasPerSm), dim3(kBulkThreads), kBulkSmem, l.stream, g, f);
+        return launch_pdl(stream_bulk_kernel<F>, dim3(l.n_sms * kBulkGridPerSm), dim3(kBulkThreads), kBulkSmem, l.stream, g, f);
     }
     return launch_pdl(stream_generic_kernel<F>, dim3(l.n_sms * kGenCtasPerSm), dim3(kGenThreads), 0, l.stream, g, f);
 }

@@ -55,9 +55,9 @@ struct Shared {
     Scalars sc;
 };
 
-// Inclusive scan over the block with ONE barrier: every thread adds up the warp totals before its own
-// warp.  `flip` (the same in every thread) alternates the two partial buffers, so the next scan may
-// write while slow threads still read this one's partials.
+// Inclusive scan over the block with ONE barrier: after it, every warp scans the (at most 32) warp totals
+// for itself with shuffles.  `flip` (the same in every thread) alternates the two partial buffers, so the
+// next scan may write while slow threads still read this one's partials.
 template <int NT>
 __device__ __forceinline__ unsigned long long scan1(unsigned long long v, unsigned long long (*part)[32], uint32_t &flip,
                                                     unsigned long long *total)
@@ -68,15 +68,10 @@ __device__ __forceinline__ unsigned long long scan1(unsigned long long v, unsign
     v = warp_incl_scan(v);
     if (lane == 31) t[wid] = v;
     __syncthreads();
-    unsigned long long off = 0, tot = 0;
-#pragma unroll
-    for (int w = 0; w < NT / 32; ++w) {
-        const unsigned long long x = t[w];
-        tot += x;
-        if (w < wid) off += x;
-    }
-    *total = tot;
-    return v + off;
+    const unsigned long long x = warp_incl_scan(lane < NT / 32 ? t[lane] : 0ull);
+    *total = __shfl_sync(0xFFFFFFFFu, x, NT / 32 - 1);
+    const unsigned long long before = __shfl_sync(0xFFFFFFFFu, x, wid ? wid - 1 : 0);
+    return v + (wid ? before : 0ull);
 }
 
 template <int NT>
@@ -88,10 +83,7 @@ __device__ __forceinline__ uint32_t min1(uint32_t v, uint32_t (*part)[32], uint3
     v = __reduce_min_sync(0xFFFFFFFFu, v);
     if (lane == 0) t[wid] = v;
     __syncthreads();
-    uint32_t m = INF;
-#pragma unroll
-    for (int w = 0; w < NT / 32; ++w) m = min(m, t[w]);
-    return m;
+    return __reduce_min_sync(0xFFFFFFFFu, lane < NT / 32 ? t[lane] : INF);
 }
 
 // Section 3.2 trigger for a shortage in pool X: the donor Y must have more than threshold_high of its units free
@@ -348,14 +340,9 @@ __device__ void step_body(const Geom &g, Shared<NT> &sh, const avmp_op *__restri
             nf0 = sc.nfree[0]; nv0 = sc.nvfree[0]; nf1 = sc.nfree[1]; nv1 = sc.nvfree[1];
             have_counts = true;
         }
-        bool fast = true;
-        uint32_t nF = 0;
-#pragma unroll
-        for (int w = 0; w < NT / 32; ++w) {
-            const uint32_t x = sh.w_shape[w];
-            fast = fast && (x >> 31);
-            nF += x & 0x7FFFFFFFu;
-        }
+        const uint32_t shape = lane < NT / 32 ? sh.w_shape[lane] : 0x80000000u;
+        const bool fast = __all_sync(0xFFFFFFFFu, (shape >> 31) != 0u);
+        const uint32_t nF = __reduce_add_sync(0xFFFFFFFFu, shape & 0x7FFFFFFFu);
 
         // ---- same-slot dependencies inside the window ----
         int prev_same = -1;        // >= 0: an earlier op of this window touches the same slot
