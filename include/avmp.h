@@ -212,8 +212,9 @@ AVMP_API int avmp_step(avmp_ctx *ctx, const avmp_op *d_ops, uint32_t n_ops, uint
 
 /* avmp_step followed by avmp_translate of d_handles against the tables that step leaves (Sections 3.1-3.2
  * and Figure 1), with the translation riding on the step's relocation-copy launch: two launches per engine
- * step instead of three, which is most of what the allocator part of a step costs.  Results are exactly those
- * of the two calls made one after the other.  n_handles == 0 is avmp_step; n_ops == 0 is avmp_translate. */
+ * step instead of three, which is most of what the allocator part of a step costs (lists of more than 32 768
+ * handles, and contexts with migration disabled, take the wide translate kernel as a third launch).  Results
+ * are exactly those of the two calls made one after the other.  n_handles == 0 is avmp_step; n_ops == 0 is avmp_translate. */
 AVMP_API int avmp_step_translate(avmp_ctx *ctx, const avmp_op *d_ops, uint32_t n_ops, uint32_t *d_status,
                                  const uint32_t *d_handles, uint32_t n_handles, uint32_t *d_pool, uint64_t *d_offset,
                                  uint64_t *d_arena_offset, void *stream);

@@ -301,19 +301,22 @@ static int step_rounds(avmp_ctx *c, const avmp_op *d_ops, uint32_t n_ops, const 
     uint32_t rounds = 1;
     if (c->opt.migration_enabled)
         rounds = (uint32_t)((n_ops - 1) / c->opt.min_rebalance_interval_ops) + 1;
+    // The copy grid is narrow (one 64-thread CTA per SM): a short handle list rides on it for free, a long one
+    // (tens of thousands of handles; measured cross-over near 50 000) is faster in the wide translate kernel.
+    const bool ride = c->opt.migration_enabled && tr.n && tr.n <= 32768u;
     for (uint32_t r = 0; r < rounds; ++r) {
         if (launch_step(c->g, d_ops, n_ops, d_n_ops, d_status, r == 0, S(stream)) != cudaSuccess) return AVMP_ECUDA;
         c->launches += 1;
         if (c->opt.migration_enabled) {
             // the last round's copy launch also carries the translation: two launches per step, not three
-            const cudaError_t e = (tr.n && r + 1 == rounds)
+            const cudaError_t e = (ride && r + 1 == rounds)
                                       ? launch_relocate_translate(c->g, tr.h, tr.n, tr.pool, tr.off, tr.aoff, L(c, stream))
                                       : launch_relocate(c->g, L(c, stream));
             if (e != cudaSuccess) return AVMP_ECUDA;
             c->launches += 1;
         }
     }
-    if (tr.n && !c->opt.migration_enabled) {
+    if (tr.n && !ride) {
         if (launch_translate(c->g, tr.h, tr.n, tr.pool, tr.off, tr.aoff, L(c, stream)) != cudaSuccess) return AVMP_ECUDA;
         c->launches += 1;
     }

@@ -126,20 +126,25 @@ struct RelocPieces {
 };
 
 // a10 for one handle: pool tag, offset inside that store, offset inside the arena.
-__device__ __forceinline__ void translate_one(const Geom &g, uint32_t hv, uint32_t i, uint32_t *__restrict__ pool,
-                                              unsigned long long *__restrict__ off, unsigned long long *__restrict__ aoff)
+__device__ __forceinline__ void translate_store(const Geom &g, uint32_t hv, uint32_t slot, uint32_t i, uint32_t *pool,
+                                                unsigned long long *off, unsigned long long *aoff)
 {
-    const uint32_t p = hv >> 31, vid = hv & 0x7FFFFFFFu;
-    uint32_t slot = kInvalid;
-    if (hv != kInvalid && vid < g.V[p]) slot = g.VT[p][vid];
     if (slot == kInvalid) {
         pool[i] = kInvalid; off[i] = kNone64;
         if (aoff) aoff[i] = kNone64;
         record_error(g.st, AVMP_DEV_BAD_HANDLE);
     } else {
+        const uint32_t p = hv >> 31;
         pool[i] = p; off[i] = (unsigned long long)slot * g.U[p];
         if (aoff) aoff[i] = (unsigned long long)(unit_ptr(g, p, slot) - g.arena);
     }
+}
+__device__ __forceinline__ void translate_one(const Geom &g, uint32_t hv, uint32_t i, uint32_t *pool,
+                                              unsigned long long *off, unsigned long long *aoff)
+{
+    const uint32_t p = hv >> 31, vid = hv & 0x7FFFFFFFu;
+    const uint32_t slot = (hv != kInvalid && vid < g.V[p]) ? g.VT[p][vid] : kInvalid;
+    translate_store(g, hv, slot, i, pool, off, aoff);
 }
 
 // a7 + a10 in one launch: the relocation copy of a step, and the translation of a handle list against the
@@ -153,8 +158,28 @@ struct RelocTranslate : RelocPieces {
     unsigned long long *off, *aoff;
     __device__ void tail(const Geom &g) const
     {
-        for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
-            translate_one(g, h[i], i, pool, off, aoff);
+        // eight handles per thread and round, their look-ups in flight together: the copy grid is small
+        // (one narrow CTA per SM), so a long list would otherwise pay two dependent reads per handle in series
+        constexpr int kPer = 8;
+        const uint32_t stride = gridDim.x * blockDim.x;
+        for (uint32_t base = blockIdx.x * blockDim.x + threadIdx.x; base < n; base += stride * kPer) {
+            uint32_t hv[kPer], slot[kPer];
+#pragma unroll
+            for (int j = 0; j < kPer; ++j) {
+                const unsigned long long i = (unsigned long long)base + (unsigned long long)j * stride;
+                hv[j] = i < n ? h[i] : kInvalid;
+            }
+#pragma unroll
+            for (int j = 0; j < kPer; ++j) {
+                const uint32_t p = hv[j] >> 31, vid = hv[j] & 0x7FFFFFFFu;
+                slot[j] = (hv[j] != kInvalid && vid < g.V[p]) ? g.VT[p][vid] : kInvalid;
+            }
+#pragma unroll
+            for (int j = 0; j < kPer; ++j) {
+                const unsigned long long i = (unsigned long long)base + (unsigned long long)j * stride;
+                if (i < n) translate_store(g, hv[j], slot[j], (uint32_t)i, pool, off, aoff);
+            }
+        }
     }
 };
 
@@ -555,9 +580,9 @@ cudaError_t launch_stream(const Geom &g, const F &f, bool bulk_ok, const Launch 
 inline bool mult16(unsigned long long x) { return (x & 15ull) == 0; }
 
 // ---- a10: translate ------------------------------------------------------------------
-__global__ void translate_kernel(const Geom g, const uint32_t *__restrict__ h, uint32_t n,
-                                 uint32_t *__restrict__ pool, unsigned long long *__restrict__ off,
-                                 unsigned long long *__restrict__ aoff)
+__global__ void translate_kernel(const Geom g, const uint32_t *h, uint32_t n,
+                                 uint32_t *pool, unsigned long long *off,
+                                 unsigned long long *aoff)
 {
     pdl_prologue();
     for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
@@ -566,8 +591,8 @@ __global__ void translate_kernel(const Geom g, const uint32_t *__restrict__ h, u
 
 // ---- a11 plan: request list -> row prefix sums (cu_seqlens) and piece prefix sums --------
 __global__ void __launch_bounds__(kStepThreads)
-kv_plan_kernel(const Geom g, const uint32_t *__restrict__ reqs, const uint32_t *__restrict__ tok_start,
-               uint32_t n, uint32_t subs, uint32_t *__restrict__ cu_out)
+kv_plan_kernel(const Geom g, const uint32_t *reqs, const uint32_t *tok_start,
+               uint32_t n, uint32_t subs, uint32_t *cu_out)
 {
     __shared__ unsigned long long tmp[32];
     unsigned long long run_rows = 0, run_items = 0, tot;

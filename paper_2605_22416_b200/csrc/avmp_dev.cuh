@@ -127,6 +127,9 @@ __device__ __forceinline__ uint32_t find_owner(const uint32_t *a, uint32_t lo, u
 // hidden), then waits until everything before it in the stream has completed and is visible.
 // No global memory is touched before the wait, so stream order is preserved exactly; launched
 // without the attribute the two instructions do nothing.
+// Because a kernel may be resident while its predecessor still writes, no kernel reads its inputs
+// through the read-only (non-coherent) path: kernel pointer parameters are not `const __restrict__`.
+// (A gather that read its plan that way saw the previous call's plan.)
 __device__ __forceinline__ void pdl_prologue()
 {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");

@@ -38,8 +38,8 @@ constexpr int kThreads = 256;
 // One CTA: held length of every request -> exclusive prefix sums of rows and of work items
 // (an item is `tpi` consecutive rows of one request).
 __global__ void __launch_bounds__(kStepThreads)
-static_plan_kernel(const Geom g, uint32_t *__restrict__ scratch, const uint32_t *__restrict__ reqs,
-                   uint32_t n, uint32_t tpi, uint32_t *__restrict__ cu_out)
+static_plan_kernel(const Geom g, uint32_t *scratch, const uint32_t *reqs,
+                   uint32_t n, uint32_t tpi, uint32_t *cu_out)
 {
     __shared__ unsigned long long tmp[32];
     unsigned long long run_rows = 0, run_items = 0, tot;
@@ -87,9 +87,9 @@ __device__ __forceinline__ void warp_copy_bytes(uint8_t *dst, const uint8_t *src
 // Warps walk the items grid-strided; rows of an item that share a page are one contiguous
 // run in the page and in the batch buffer.
 __global__ void __launch_bounds__(kThreads)
-static_gather_kernel(const Geom g, const uint32_t *__restrict__ scratch, const uint32_t layer,
-                     const uint32_t *__restrict__ reqs, const uint32_t n, const uint32_t tpi,
-                     uint8_t *__restrict__ out_k, uint8_t *__restrict__ out_v, const unsigned long long cap_tokens)
+static_gather_kernel(const Geom g, const uint32_t *scratch, const uint32_t layer,
+                     const uint32_t *reqs, const uint32_t n, const uint32_t tpi,
+                     uint8_t *out_k, uint8_t *out_v, const unsigned long long cap_tokens)
 {
     pdl_prologue();
     const uint32_t *cu_rows = scratch + kRowsOff, *cu_items = scratch + kItemsOff;

@@ -27,8 +27,8 @@ using namespace stepimpl;
 
 template <int NT>
 __global__ void __launch_bounds__(NT, 1)
-step_kernel(const Geom g, const avmp_op *__restrict__ ops, const uint32_t n_ops_max,
-            const uint32_t *__restrict__ n_ops_dev, uint32_t *__restrict__ status, const int first_round)
+step_kernel(const Geom g, const avmp_op *ops, const uint32_t n_ops_max,
+            const uint32_t *n_ops_dev, uint32_t *status, const int first_round)
 {
     __shared__ Shared<NT> sh;
     pdl_prologue();

@@ -236,8 +236,8 @@ __device__ __forceinline__ void pop_units(const Geom &g, Shared<NT> &sh, uint32_
 // The whole allocator update for ops[0 .. n_ops) by the calling CTA of NT threads (callers have
 // already waited for everything earlier in the stream).
 template <int NT>
-__device__ void step_body(const Geom &g, Shared<NT> &sh, const avmp_op *__restrict__ ops, const uint32_t n_ops,
-                          uint32_t *__restrict__ status, const int first_round)
+__device__ void step_body(const Geom &g, Shared<NT> &sh, const avmp_op *ops, const uint32_t n_ops,
+                          uint32_t *status, const int first_round)
 {
     constexpr uint32_t kHash = Shared<NT>::kHash;
     Scalars &sc = sh.sc;

@@ -2,7 +2,7 @@
 a handful of launches): `python tests/profile_case.py <case>`.  Measurement tooling, not part of the library.
 
 Cases: ssm_gather, kv_gather (one layer per launch), ssm_gather_fused, kv_gather_fused (several
-layers per launch), relocate, step.  Every case builds a context through the
+layers per launch), step_gather (both kinds, all layers, one launch), relocate, step.  Every case builds a context through the
 C ABI, brings it to a busy state with a few allocator steps and then launches the kernel
 of interest `--repeat` times on different layers, so every launch reads cold data.
 """
@@ -28,7 +28,7 @@ def _dev(a):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["ssm_gather", "kv_gather", "ssm_gather_fused", "kv_gather_fused", "relocate", "step"])
+    ap.add_argument("case", choices=["ssm_gather", "kv_gather", "ssm_gather_fused", "kv_gather_fused", "step_gather", "relocate", "step"])
     ap.add_argument("--repeat", type=int, default=6)
     ap.add_argument("--pool-gib", type=float, default=3.0)
     ap.add_argument("--layers", type=int, default=8, help="layers per launch in the fused cases")
@@ -36,6 +36,37 @@ def main():
     m = W.JAMBA_LIKE
     pool = int(args.pool_gib * W.GiB)
     ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    if args.case == "step_gather":
+        # a small engine step: 40 requests x 600 tokens, every attention and SSM layer in ONE launch
+        n_req, tokens = 40, 600
+        ctx = B.Context(m, pool, 0.6, 128, max_requests=256, max_pages=256)
+        s0 = ctx.stats()
+        n_req = min(n_req, s0["cap_ssm"] // m.n_ssm_layers, s0["cap_kv"] // (tokens // 16 + 1))
+        st = np.zeros(n_req, np.uint32)
+        ctx.step_host(W.make_ops(W.OP_ADMIT, np.arange(n_req), tokens), n_req, st)
+        assert (st == 0).all(), st
+        reqs = _dev(np.random.default_rng(0).permutation(n_req).astype(np.uint32))
+        tot = n_req * tokens
+        cu = torch.zeros(n_req + 1, dtype=torch.int32, device="cuda")
+        bufs = [(torch.empty((m.n_attn_layers, tot, m.kv_row_bytes), dtype=torch.uint8, device="cuda"),
+                 torch.empty((m.n_attn_layers, tot, m.kv_row_bytes), dtype=torch.uint8, device="cuda"),
+                 torch.empty((m.n_ssm_layers, n_req, m.state_bytes), dtype=torch.uint8, device="cuda"),
+                 torch.empty((m.n_ssm_layers, n_req, m.conv_bytes), dtype=torch.uint8, device="cuda")) for _ in range(2)]
+        nbytes = 2 * tot * 2 * m.kv_row_bytes * m.n_attn_layers + 2 * n_req * (m.state_bytes + m.conv_bytes) * m.n_ssm_layers
+        for i in range(args.repeat):
+            ok, ov, os_, oc = bufs[i % 2]
+            a, b = ev(), ev()
+            a.record()
+            ctx.gather_step(reqs, n_req, 0, m.n_attn_layers, ok, ov, tot * m.kv_row_bytes, tot, cu,
+                            0, m.n_ssm_layers, os_, n_req * m.state_bytes, oc, n_req * m.conv_bytes)
+            b.record()
+            torch.cuda.synchronize()
+            print(f"step_gather launch {i}: {a.elapsed_time(b) * 1e3:.1f} us, {nbytes / 1e6:.0f} MB, "
+                  f"{nbytes / a.elapsed_time(b) / 1e6:.0f} GB/s")
+        print(ctx.stats())
+        ctx.close()
+        return
 
     if args.case in ("ssm_gather_fused", "kv_gather_fused"):
         kv = args.case == "kv_gather_fused"
