@@ -76,11 +76,12 @@ struct SsmPieces {
         const uint32_t dl = (uint32_t)(it / per_layer);
         const uint32_t rem = (uint32_t)(it % per_layer);
         const uint32_t k = rem / per, c = rem % per;
-        const uint32_t r = reqs[k];
+        const unsigned long long keep = l2_policy_evict_last();
+        const uint32_t r = ld_keep(reqs + k, keep);
         uint32_t slot = kInvalid;
-        if (r < g.R && g.r_state[r] == AVMP_REQ_LIVE) {
-            const uint32_t h = g.r_ssm[(unsigned long long)r * g.ns + layer0 + dl];
-            if (h != kInvalid) slot = g.VT[1][h & 0x7FFFFFFFu];
+        if (r < g.R && ld_keep(g.r_state + r, keep) == AVMP_REQ_LIVE) {
+            const uint32_t h = ld_keep(g.r_ssm + ((unsigned long long)r * g.ns + layer0 + dl), keep);
+            if (h != kInvalid) slot = ld_keep(g.VT[1] + (h & 0x7FFFFFFFu), keep);
         }
         if (slot == kInvalid) {
             if (c == 0) record_error(g.st, AVMP_DEV_BAD_REQUEST);
@@ -234,19 +235,20 @@ struct KvPieces {
         // of a round (two dependent reads per entry) are in flight together; taken one entry at a time
         // between barriers they would cost that latency once per entry.
         constexpr int kPer = 8;
+        const unsigned long long keep = l2_policy_evict_last();
         for (uint32_t base = 0; base < n; base += kPer * blockDim.x) {
             uint32_t rr[kPer], t0[kPer], st[kPer], ln[kPer];
 #pragma unroll
             for (int i = 0; i < kPer; ++i) {
                 const uint32_t k = base + threadIdx.x + i * blockDim.x;
-                rr[i] = k < n ? reqs[k] : kInvalid;
+                rr[i] = k < n ? ld_keep(reqs + k, keep) : kInvalid;
                 t0[i] = (k < n && tok_start) ? tok_start[k] : 0u;
             }
 #pragma unroll
             for (int i = 0; i < kPer; ++i) {
                 const bool in_range = rr[i] < g.R;
-                st[i] = in_range ? g.r_state[rr[i]] : (uint32_t)AVMP_REQ_EMPTY;
-                ln[i] = in_range ? g.r_len[rr[i]] : 0u;
+                st[i] = in_range ? ld_keep(g.r_state + rr[i], keep) : (uint32_t)AVMP_REQ_EMPTY;
+                ln[i] = in_range ? ld_keep(g.r_len + rr[i], keep) : 0u;
             }
 #pragma unroll
             for (int i = 0; i < kPer; ++i) {
@@ -304,8 +306,9 @@ struct KvPieces {
         const uint32_t b_hi = min((hi_t - page * T) * row, (q + 1u) * kStage);
         if (b_lo >= b_hi) return Piece{nullptr, nullptr, 0};
         const uint32_t r = req_of[k];
-        const uint32_t h = g.r_chain[(unsigned long long)r * g.max_pages + page];
-        const uint32_t slot = g.VT[0][h & 0x7FFFFFFFu];
+        const unsigned long long keep = l2_policy_evict_last();
+        const uint32_t h = ld_keep(g.r_chain + ((unsigned long long)r * g.max_pages + page), keep);
+        const uint32_t slot = ld_keep(g.VT[0] + (h & 0x7FFFFFFFu), keep);
         uint8_t *p = g.arena + (unsigned long long)slot * g.U[0] + (unsigned long long)(layer0 + dl) * g.kv_layer_bytes +
                      (unsigned long long)part * T * row + b_lo;
         // byte b of the page part is byte (b - (t0 - page*T)*row) of the request's rows

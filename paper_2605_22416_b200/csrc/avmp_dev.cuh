@@ -66,6 +66,23 @@ __device__ __forceinline__ void record_error(DevState *st, unsigned long long co
     atomicAdd(&st->error_count, 1ull);
 }
 
+// Table reads of the copy kernels (request list, request records, chains, page table): a few KB that every
+// launch needs first, in the middle of GBs of payload streaming through L2.  They are read with an L2
+// evict-last policy so that the next launch finds them in L2 instead of paying DRAM latency three or four
+// times in a row before its first copy can be issued.
+__device__ __forceinline__ unsigned long long l2_policy_evict_last()
+{
+    unsigned long long p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint32_t ld_keep(const uint32_t *ptr, unsigned long long policy)
+{
+    uint32_t v;
+    asm volatile("ld.global.L2::cache_hint.u32 %0, [%1], %2;" : "=r"(v) : "l"(ptr), "l"(policy) : "memory");
+    return v;
+}
+
 // ---- warp / block primitives (blockDim.x == kStepThreads for the block ones) ----
 __device__ __forceinline__ unsigned long long warp_incl_scan(unsigned long long v)
 {
