@@ -639,3 +639,25 @@ def random_op_string(seed: int, n: int, max_requests: int, max_tokens: int,
     ops["req"] = req
     ops["tokens"] = tok
     return ops
+
+
+def engine_shaped_batch(seed: int, max_requests: int, max_tokens: int, p_pick: float = 0.5,
+                        repeats: bool = False) -> np.ndarray:
+    """One batch in the order an engine step has -- FINISH ops, then EXTEND ops, then ADMIT ops, slots ascending
+    inside each kind -- but with the slots of each kind drawn independently, so the same slot may be finished and
+    admitted (or extended) in one batch, finished with KEEP_KV and resumed, or extended and admitted: the cases a
+    scheduler never emits and an allocator must still get right.  repeats: some ops appear twice in a row (the
+    second one sees what the first one did), which breaks the ascending order by the smallest possible margin."""
+    parts = []
+    for j, kind in enumerate((OP_FINISH, OP_EXTEND, OP_ADMIT)):
+        u = rand_unit(seed, 31 + j, max_requests)
+        slots = np.flatnonzero(u < p_pick * (0.6 if kind == OP_FINISH else 1.0))
+        n = len(slots)
+        tok = rand_int(seed, 41 + j, n, 1, max_tokens) if n else np.zeros(0, np.int64)
+        fl = rand_int(seed, 51 + j, n, 0, 3) if n else np.zeros(0, np.int64)
+        flags = (fl & FLAG_KEEP_KV) if kind == OP_FINISH else ((fl & FLAG_RESUME) if kind == OP_ADMIT else 0 * fl)
+        part = make_ops(kind, slots, tok, flags)
+        if repeats and n:
+            part = np.repeat(part, np.where(rand_unit(seed, 61 + j, n) < 0.15, 2, 1))
+        parts.append(part)
+    return np.concatenate(parts)

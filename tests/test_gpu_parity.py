@@ -1051,3 +1051,41 @@ def test_step_translate_equals_step_then_translate(env, name, steps, over):
     assert seen["handles"] > 500 and seen["dead"] > 0
     if w.migration_enabled:
         assert g.stats()["n_rebalance"] > 0
+
+
+@pytest.mark.parametrize("case,slots,pool_kib,interval,tokens", [
+    (0, 8, 1, 4, 40),            # the hand-sized pool: shortages and migrations in most batches
+    (1, 40, 6, 7, 60),
+    (2, 300, 40_000, 100, 200),  # two windows of 256 ops: the shape is judged per window
+    (3, 300, 2_000, 50, 200),    # the same, tight
+    (4, 1500, 12_000, 300, 120), # 1024-op windows; tight enough for OOM storms
+    (5, 1500, 400_000, 1000, 120),
+])
+def test_engine_shaped_batches_with_shared_slots(env, case, slots, pool_kib, interval, tokens):
+    """Batches in an engine step's order (FINISH*, EXTEND*, ADMIT*, ascending slots inside a kind -- the shape the
+    step kernel recognises and handles without its same-slot table) whose kinds share slots: finished and admitted
+    again in one batch, parked with KEEP_KV and resumed, extended and admitted; every third batch also repeats some
+    ops back to back (equal slots inside a kind: no longer that shape).  Statuses and every table against the
+    oracle after every batch."""
+    model = W.TINY_MODEL if case < 2 else W.SMALL_UNIT_MODEL
+    w = W.Workload(f"shaped{case}", model, pool_kib * 1024, 0.5, 1 + case % 3 if case < 2 else 16 * (1 + case % 3),
+                   slots, slots, 16, "queue", 0, min_rebalance_interval_ops=interval, reclaim_gap=bool(case % 2))
+    g, o = _pair(env, w)
+    rounds = 120 if slots <= 300 else 40
+    shortages = 0
+    for rnd in range(rounds):
+        ops = W.engine_shaped_batch(1000 * case + rnd, slots, tokens, p_pick=0.25 + 0.5 * ((rnd * 7) % 10) / 10,
+                                    repeats=rnd % 3 == 2)
+        if len(ops) == 0:
+            continue
+        sg, so = g.step(ops), o.step(ops)
+        assert np.array_equal(sg, so), (case, rnd, np.flatnonzero(sg != so)[:10], sg[sg != so][:10], so[sg != so][:10])
+        shortages += int((so == W.ST_OOM).sum())
+        if rnd % 4 == 0 or slots <= 40:
+            env["same"](g, o, w, f"case {case} round {rnd}")
+    env["same"](g, o, w, "end")
+    s = g.stats()
+    check_invariants(s, g.tables(), page_tokens=16, n_ssm_layers=model.n_ssm_layers, max_pages=16)
+    assert s["n_invalid"] > 0                      # shared slots make some ops BAD_REQ, as they must
+    if case in (0, 1, 3, 4):
+        assert shortages > 0 and s["n_rebalance"] > 0
