@@ -564,3 +564,33 @@ def test_bytes_inside_a_unit_follow_the_documented_layout(shape):
     seen = check_unit_layout(w, o, read_units)
     assert seen["kv_rows"] > 1000 and seen["ssm_blocks"] > 40 and seen["relocated_blocks"] > 4
     _inv(o, w)
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_naive_model_on_engine_shaped_batches(seed):
+    """The same brute-force comparison on batches in an engine step's order whose kinds share slots (finished and
+    admitted again, parked and resumed, extended and admitted in one batch) and repeat ops back to back: the
+    sequences the GPU path's window-shape shortcut must get right are pinned on the oracle side too."""
+    w = W.config("tiny", migration_batch_size=1 + seed % 3, min_rebalance_interval_ops=3 + seed)
+    o = Oracle.from_workload(w, max_requests=6, max_pages=8)
+    nv = M.NaiveAllocator(w.model, w.pool_bytes, w.split, w.migration_batch_size, 6, 8,
+                          min_interval=w.min_rebalance_interval_ops)
+    for rnd in range(60):
+        ops = W.engine_shaped_batch(77 * seed + rnd, 6, 50, p_pick=0.3 + 0.05 * (rnd % 8), repeats=rnd % 3 == 2)
+        st = o.step(ops)
+        for i in range(len(ops)):
+            ex = nv.op(int(ops["kind"][i]), int(ops["flags"][i]), int(ops["req"][i]), int(ops["tokens"][i]))
+            assert int(st[i]) == ex, (rnd, i, ops[i])
+        t = o.tables()
+        chain = t["req_chain"].reshape(6, 8)
+        for r in range(6):
+            q = nv.reqs[r]
+            assert int(t["req_state"][r]) == q.state and int(t["req_len"][r]) == q.length
+            assert chain[r, :len(q.chain)].tolist() == q.chain
+        for p, nm in enumerate(("kv", "ssm")):
+            assert t[f"slot_stack_{nm}"][::-1].tolist() == nv.next_slots[p]
+            assert t[f"vid_stack_{nm}"][::-1].tolist() == nv.next_ids[p]
+        s = o.stats()
+        assert (s["cap_kv"], s["cap_ssm"]) == tuple(nv.cap) and s["n_oom"] == nv.n_oom and s["n_rebalance"] == nv.n_rebalance
+        _inv(o, w.with_(max_pages=8))
+    assert o.stats()["n_rebalance"] > 0 and o.stats()["n_oom"] > 0
