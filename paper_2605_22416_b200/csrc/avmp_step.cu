@@ -1,19 +1,23 @@
 // avmp_step: the batched allocator update (paper Sections 3.1-3.2) as one planning CTA.
 //
 // The batch must behave exactly as if its ops were applied one at a time.  The CTA cuts
-// the batch into windows of 1024 ops (one per thread) and each window into maximal runs of
-// ops that point the same way (all FINISH, or all ADMIT/EXTEND) and touch distinct request
-// slots.  Inside a run the sequential result has a closed form:
+// the batch into windows of NT ops (one per thread; NT = 256, 512 or 1024 by batch length)
+// and each window into maximal runs of ops that point the same way (all FINISH, or all
+// ADMIT/EXTEND) and touch distinct request slots.  Inside a run the sequential result has a
+// closed form:
 //   * free run  -- an exclusive prefix sum of the units each op releases gives the stack
 //                  position of every pushed slot and id;
-//   (same-slot repeats inside a window are found with a shared-memory hash of the slots)
 //   * alloc run -- an exclusive prefix sum of the demands gives the stack entries every op
 //                  pops, as long as every op before it fits.  The first op whose inclusive
 //                  demand exceeds the free count is the first sequential failure: everything
 //                  before it is committed, the CapacityError handler (Section 3.2) runs for
-//                  that op alone with the whole CTA helping (stack compaction, relocation
-//                  list, recipient growth), the op is retried once, and the scan resumes
-//                  behind it.  A failed op takes nothing, so the same prefix sums stay valid.
+//                  that op alone (a migration with the whole CTA helping: stack compaction,
+//                  relocation list, recipient growth), the op is retried once, and the scan
+//                  resumes behind it.  A failed op takes nothing, so the same prefix sums
+//                  stay valid.
+// A window in an engine step's order (FINISH*, EXTEND*, ADMIT*, ascending slots inside a kind)
+// is recognised with one ballot per warp and has exactly those two runs; any other window finds
+// its runs through a shared-memory hash of the slots (avmp_step_body.cuh).
 // Relocated payload is copied by a separate wide kernel after this one, so a launch performs
 // at most one migration; if a second one is due, the launch stops before that op and the
 // host-queued next round resumes there (the throttle bounds the number of rounds).
