@@ -526,7 +526,11 @@ def other_configs(dev, skip: str) -> list:
         if name == skip:
             continue
         w = W.config(name)
-        res = measure(w, dev, steps=k, warmup=3, warm_steps=ws, asked_lpl=0, full=False)
+        try:
+            res = measure(w, dev, steps=k, warmup=3, warm_steps=ws, asked_lpl=0, full=False)
+        except Exception as exc:      # a side measurement must not take the headline line down with it
+            rows.append({"workload": name, "unavailable": f"{type(exc).__name__}: {exc}"})
+            continue
         f = class_figures(res, w.model, peak)
         rows.append({"workload": name, "steps": res["K"], "timed_region_ms": res["total_ms"],
                      "value": res["moved"] / (res["total_ms"] * 1e-3) / 1e9, "frac": res["moved"] / (res["total_ms"] * 1e-3) / 1e9 / peak,
@@ -994,16 +998,24 @@ def main():
             import torch
             dev = torch.device("cuda", local_rank)
             sec = out["roofline"]["secondary"]
-            sec["relocation_copy"] = migration_microbench(dev)
-            sec["allocator_vs_step_batch"] = allocator_scaling(dev)
-            sec["write_side"] = write_side_microbench(dev)
+            for key, fn in (("relocation_copy", migration_microbench), ("allocator_vs_step_batch", allocator_scaling),
+                            ("write_side", write_side_microbench)):
+                try:
+                    sec[key] = fn(dev)
+                except Exception as exc:      # side measurements must not take the headline line down with them
+                    sec[key] = {"unavailable": f"{type(exc).__name__}: {exc}"}
             try:
                 sec["remap_vs_copy"] = {"remap": remap_microbench(dev), "copy": relocation_small_cases(dev)}
             except Exception as exc:          # the comparison is context for one design decision, not part of the path
                 sec["remap_vs_copy"] = {"unavailable": f"{type(exc).__name__}: {exc}"}
-            sec["closed_loop_device"] = device_closed_loop(dev, args.workload, 1500 if args.workload == "scale" else 3000)
+            try:
+                sec["closed_loop_device"] = device_closed_loop(dev, args.workload, 1500 if args.workload == "scale" else 3000)
+            except Exception as exc:
+                sec["closed_loop_device"] = {"unavailable": f"{type(exc).__name__}: {exc}"}
             out["roofline"]["other_configs"] = other_configs(dev, skip=args.workload)
         if not args.no_cpu_baseline:
+            import torch
+            torch.cuda.empty_cache()
             out["cpu_baseline"] = run_oracle(args, n_sample_steps=12)
         print(json.dumps(out), flush=True)
     if world > 1:
