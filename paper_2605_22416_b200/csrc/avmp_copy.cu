@@ -79,9 +79,11 @@ struct SsmPieces {
         const unsigned long long keep = l2_policy_evict_last();
         const uint32_t r = ld_keep(reqs + k, keep);
         uint32_t slot = kInvalid;
-        if (r < g.R && ld_keep(g.r_state + r, keep) == AVMP_REQ_LIVE) {
+        if (r < g.R) {
+            // state and handle are read together: one round trip less on the way to the first copy
+            const uint32_t state = ld_keep(g.r_state + r, keep);
             const uint32_t h = ld_keep(g.r_ssm + ((unsigned long long)r * g.ns + layer0 + dl), keep);
-            if (h != kInvalid) slot = ld_keep(g.VT[1] + (h & 0x7FFFFFFFu), keep);
+            if (state == AVMP_REQ_LIVE && h != kInvalid) slot = ld_keep(g.VT[1] + (h & 0x7FFFFFFFu), keep);
         }
         if (slot == kInvalid) {
             if (c == 0) record_error(g.st, AVMP_DEV_BAD_REQUEST);
