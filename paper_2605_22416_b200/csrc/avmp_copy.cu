@@ -233,18 +233,21 @@ struct KvPieces {
         if (n > kLocalPlanMax) { cu_items = g.g_cu_items; cu_rows = g.g_cu_rows; req_of = reqs; return; }
         uint32_t *rows_s = buf, *items_s = buf + kLocalPlanMax + 1, *req_s = buf + 2 * (kLocalPlanMax + 1);
         const bool lead = blockIdx.x == 0;            // one CTA reports errors and writes cu_seqlens
-        // Pass 1: every entry's rows and pieces.  Eight entries per thread and round, so that the table reads
-        // of a round (two dependent reads per entry) are in flight together; taken one entry at a time
-        // between barriers they would cost that latency once per entry.
+        // Every thread takes a run of consecutive entries: their rows and pieces (eight entries per round, so
+        // that the two dependent table reads of a round are in flight together), summed on the way; ONE block
+        // scan orders the runs; then each thread turns its own entries into exclusive prefix sums in place.
         constexpr int kPer = 8;
         const unsigned long long keep = l2_policy_evict_last();
-        for (uint32_t base = 0; base < n; base += kPer * blockDim.x) {
+        const uint32_t per = (n + blockDim.x - 1) / blockDim.x;
+        const uint32_t k0 = min(n, threadIdx.x * per), k1 = min(n, k0 + per);
+        unsigned long long mine = 0, tot;
+        for (uint32_t kb = k0; kb < k1; kb += kPer) {
             uint32_t rr[kPer], t0[kPer], st[kPer], ln[kPer];
 #pragma unroll
             for (int i = 0; i < kPer; ++i) {
-                const uint32_t k = base + threadIdx.x + i * blockDim.x;
-                rr[i] = k < n ? ld_keep(reqs + k, keep) : kInvalid;
-                t0[i] = (k < n && tok_start) ? tok_start[k] : 0u;
+                const uint32_t k = kb + i;
+                rr[i] = k < k1 ? ld_keep(reqs + k, keep) : kInvalid;
+                t0[i] = (k < k1 && tok_start) ? tok_start[k] : 0u;
             }
 #pragma unroll
             for (int i = 0; i < kPer; ++i) {
@@ -254,21 +257,15 @@ struct KvPieces {
             }
 #pragma unroll
             for (int i = 0; i < kPer; ++i) {
-                const uint32_t k = base + threadIdx.x + i * blockDim.x;
-                if (k < n) {
+                const uint32_t k = kb + i;
+                if (k < k1) {
                     uint32_t rows, items;
                     kv_rows_items(g, st[i], ln[i], t0[i], subs, lead, rows, items);
                     rows_s[k] = rows; items_s[k] = items; req_s[k] = rr[i];
+                    mine += ((unsigned long long)items << 32) | rows;
                 }
             }
         }
-        __syncthreads();
-        // Pass 2: exclusive prefix sums over the list: every thread sums a run of consecutive entries,
-        // one block scan orders the runs (one scan for the whole list instead of one per window).
-        const uint32_t per = (n + blockDim.x - 1) / blockDim.x;
-        const uint32_t k0 = threadIdx.x * per, k1 = min(n, k0 + per);
-        unsigned long long mine = 0, tot;
-        for (uint32_t k = k0; k < k1; ++k) mine += ((unsigned long long)items_s[k] << 32) | rows_s[k];
         const unsigned long long incl = block_incl_scan(mine, tmp, &tot);
         unsigned long long run = incl - mine;
         for (uint32_t k = k0; k < k1; ++k) {
