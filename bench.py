@@ -36,8 +36,8 @@ from paper_2605_22416_b200 import workloads as W  # noqa: E402
 
 METRIC = "paged gather+migration GB/s over whole engine steps (allocator ops/s reported beside it)"
 WARM_STEPS = 600          # closed-loop steps before the measured window (steady state)
-# DRAM traffic of one launch of the dominant kernel, from ncu captures of this kernel (profiles/
-# ssm_gather_fused_jamba_like.md at 1 GB per launch, profiles/bench_short_uniform_dram_traffic.md at 6.8 GB):
+# DRAM traffic of one launch of the dominant kernel, from ncu captures of this kernel at 1 GB and at 6.8 GB per
+# launch (summarised under profiles/):
 # reads equal the algorithmic read bytes, and of the writes about 47 MB are still dirty in L2 when the kernel
 # ends (they reach DRAM during the next kernel).  Recorded from those captures, not re-measured per run.
 L2_DIRTY_TAIL_BYTES = 47e6
